@@ -1,0 +1,165 @@
+/* mixaq.h -- C ABI of the B200 (sm_100a) library for the quantized Two-Branch Swin Block forward of MixA-Q.
+ *
+ * What one block call computes (MixA-Q Section 3.1 "Replace Pruning with MP Execution", Section 3.2
+ * "Two-Branch Swin Block", Section 3.4 "Activation Pruning Incorporation"):
+ *   1. the feature map is cut into non-overlapping ws x ws windows, after an optional cyclic shift;
+ *   2. every window gets an importance score (squared L2 norm of its int8 score codes); per image the
+ *      windows are ranked by (score descending, window index ascending); the top ones go to the
+ *      high-precision branch, the next ones to the low-precision branch, and (optionally) the lowest ones are
+ *      pruned, i.e. forwarded unchanged;
+ *   3. each branch runs LN -> window attention -> LN -> FFN on its windows with the SAME integer weights
+ *      ("shadow layers") but its own LayerNorm parameters, step sizes, zero points and activation bit width;
+ *      all matrix products are integer with int32 accumulation;
+ *   4. results are dequantized and scattered back to the un-shifted, un-padded feature map.
+ *
+ * Conventions
+ *   - Every pointer inside the *_params structs, x, y, stage outputs, selections, taps and workspaces is a
+ *     DEVICE pointer owned by the caller.  The library never frees them and keeps none past the call, with
+ *     one exception: `prepared` buffers are read by every later forward call that gets the same params.
+ *   - Feature maps are [B][H][W][C] binary32, channels contiguous.  C must be a multiple of 32, C/heads
+ *     must be 32, window must be 7, hidden must be a multiple of 32.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*); they allocate nothing and do
+ *     not synchronise.  Errors found on the host are returned before anything is launched.
+ *   - Activation codes are unsigned, `bits` in {8, 4, 2}.  Sub-byte codes are stored bit-packed, little end
+ *     first: element e of a row lives in byte e*bits/8 at bit (e*bits) mod 8.
+ *   - There is no CPU fallback: without a CUDA device every entry point returns MIXAQ_CUDA_ERROR.
+ */
+#ifndef MIXAQ_H
+#define MIXAQ_H
+#include <stddef.h>
+#include <stdint.h>
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int mixaq_status;
+#define MIXAQ_OK                    0
+#define MIXAQ_INVALID_ARG          (-1)  /* null pointer, ratio outside [0,1], bad bit width ...          */
+#define MIXAQ_UNSUPPORTED_SHAPE    (-2)  /* window != 7, C % 32 != 0, C/heads != 32, shift >= window ...  */
+#define MIXAQ_WORKSPACE_TOO_SMALL  (-3)
+#define MIXAQ_CUDA_ERROR           (-4)  /* a CUDA runtime/driver call failed; see mixaq_last_error()     */
+#define MIXAQ_DEVICE_TIMEOUT       (-5)  /* a bounded wait inside a kernel ran out (status word)          */
+#define MIXAQ_INTERNAL             (-6)
+
+typedef struct mixaq_ctx mixaq_ctx;
+
+/* Per-tensor asymmetric activation quantizer (Section 3.2: "independent step sizes and zero points"):
+ * q = clamp(rne(x * inv_scale) + zero_point, 0, 2^bits - 1);  x ~ (q - zero_point) * scale. */
+typedef struct { int bits; float scale; float inv_scale; int zero_point; } mixaq_aq;
+
+/* Integer weight matrix shared by both branches: signed codes, one per byte, row-major [out][in];
+ * per-output-channel step size.  `bits` documents the code range (|code| <= 2^(bits-1)-1). */
+typedef struct { const int8_t* codes; const float* scale; int out_features; int in_features; int bits; } mixaq_linear;
+
+/* One branch of a block: private LayerNorms, biases (may alias the other branch's), quantizers.
+ * The attention-probability quantizer is implied: `bits` bits, zero point 0, step 1/(2^bits - 1). */
+typedef struct {
+  const float *ln1_g, *ln1_b, *ln2_g, *ln2_b;
+  const float *b_qkv, *b_proj, *b_fc1, *b_fc2;
+  mixaq_aq qkv_in, q, k, v, proj_in, fc1_in, fc2_in;
+  int bits;
+} mixaq_branch;
+
+typedef struct {
+  int dim, heads, window, shift, hidden;
+  mixaq_linear qkv, proj, fc1, fc2;       /* [3C][C], [C][C], [hidden][C], [C][hidden]                    */
+  const float* relpos_table;              /* [(2*window-1)^2][heads] binary32                              */
+  mixaq_branch hi, lo;
+  float score_inv_scale;                  /* score code = clamp(rne(x * score_inv_scale), -127, 127)       */
+  void* prepared;                         /* device buffer of mixaq_block_prepared_bytes(), filled once by */
+                                          /* mixaq_block_prepare(); read by every forward call             */
+} mixaq_block_params;
+
+/* Patch merging between stages: 2x2 neighbours concatenated (zero padding for odd sizes) -> LN(4C) ->
+ * quantize (`in`) -> integer GEMM with `reduction` [2C][4C], no bias.  (The paper's "downsampling layers",
+ * Appendix 6.2: their cost is not reduced by the method.) */
+typedef struct { const float *ln_g, *ln_b; mixaq_aq in; mixaq_linear reduction; void* prepared; } mixaq_merge_params;
+
+typedef struct {
+  const int32_t* energy;   /* optional [B][H][W] token energies computed at stage entry (Section 3.2: the score is
+                              computed once per stage and shared); NULL: score this block's own input x      */
+  int reverse;             /* 0: highest scores go high.  1: worst-case order (Table 4): lowest scores go high */
+} mixaq_select_opts;
+
+/* Optional selection outputs (each pointer may be NULL). */
+typedef struct {
+  uint8_t* cls;            /* [B][nW]  0 high, 1 low, 2 pruned                                              */
+  int32_t* order;          /* [B][nW]  window index by rank: first n_hi high, next n_lo low, last n_pr pruned */
+  int64_t* score;          /* [B][nW]  window scores                                                         */
+} mixaq_selection;
+
+/* Optional debug taps of one branch (each pointer may be NULL).  Rows are in window-batch order: window slot
+ * s = image * n_branch + rank-within-branch, row = s*49 + in-window token.  Code tensors are bit-packed at the
+ * branch's bit width; accumulators are zero-point corrected int32. */
+typedef struct {
+  uint8_t* a_codes;   int32_t* qkv_acc;  uint8_t* qkv_codes;
+  uint8_t* p_codes;   /* [slots][heads][49][49], one code per byte */
+  int32_t* pv_acc;    uint8_t* o_codes;  int32_t* proj_acc;  float* x1;
+  uint8_t* f1_codes;  int32_t* fc1_acc;  uint8_t* f2_codes;  int32_t* fc2_acc;
+} mixaq_branch_taps;
+typedef struct { mixaq_branch_taps hi, lo; } mixaq_taps;
+
+typedef struct {
+  int num_stages;
+  const int* depths;                    /* HOST array [num_stages]; every depth is even or 1                */
+  const mixaq_block_params* blocks;     /* HOST array, sum(depths) entries                                  */
+  const mixaq_merge_params* merges;     /* HOST array, num_stages-1 entries                                 */
+} mixaq_backbone_params;
+
+/* ---- context ---- */
+/* Creates a context on `device` (makes it current).  Holds the status word and cached TMA descriptors. */
+mixaq_status mixaq_create(mixaq_ctx** ctx, int device);
+mixaq_status mixaq_destroy(mixaq_ctx* ctx);
+/* Text of the last host-side error of this context (static storage, valid until the next call). */
+const char*  mixaq_last_error(const mixaq_ctx* ctx);
+/* Reads the device status word (synchronises `cuda_stream`): MIXAQ_OK or MIXAQ_DEVICE_TIMEOUT. */
+mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream);
+
+/* ---- the one definition of "how many windows does a ratio take out of n": floor(ratio*n + 1e-6) ---- */
+int          mixaq_low_count(float ratio, int n);
+/* counts[3] = {n_hi, n_lo, n_pr} per image for an H x W map: n_pr = cnt(prune, nW), n_lo = cnt(low, nW-n_pr). */
+mixaq_status mixaq_branch_counts(int H, int W, int window, float low_ratio, float prune_ratio, int* counts);
+
+/* ---- one-time preparation of derived tables (column sums for the zero-point correction, step-size
+ *      products, expanded relative-position bias).  Asynchronous on the stream. ---- */
+size_t       mixaq_block_prepared_bytes(const mixaq_block_params* p);
+mixaq_status mixaq_block_prepare(mixaq_ctx* ctx, const mixaq_block_params* p, void* cuda_stream);
+size_t       mixaq_merge_prepared_bytes(const mixaq_merge_params* p);
+mixaq_status mixaq_merge_prepare(mixaq_ctx* ctx, const mixaq_merge_params* p, void* cuda_stream);
+
+/* ---- stage-entry scoring (Section 3.2): energy[b][y][x] = sum_c code(x[b][y][x][c])^2 ---- */
+mixaq_status mixaq_stage_energy(mixaq_ctx* ctx, const float* x, int32_t* energy, int B, int H, int W, int C,
+                                float score_inv_scale, void* cuda_stream);
+
+/* ---- one Two-Branch Swin Block (Section 3.2, Figure 3).  x and y must not overlap. ---- */
+size_t       mixaq_block_workspace_bytes(const mixaq_block_params* p, int B, int H, int W);
+mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p,
+                                 const float* x, float* y, int B, int H, int W,
+                                 float low_ratio, float prune_ratio,
+                                 const mixaq_select_opts* opts /* nullable */,
+                                 const mixaq_selection* sel_out /* nullable */,
+                                 void* workspace, size_t workspace_bytes,
+                                 const mixaq_taps* taps /* nullable */, void* cuda_stream);
+
+/* ---- patch merging alone: x [B][H][W][C] -> y [B][ceil(H/2)][ceil(W/2)][2C] ---- */
+size_t       mixaq_merge_workspace_bytes(const mixaq_merge_params* p, int B, int H, int W);
+mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
+                                 int B, int H, int W, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- the backbone: for every stage [merge] -> stage energy -> blocks; one ratio per pair of consecutive
+ *      blocks (Section 3.3), optional prune ratio per pair (Section 3.4).  x0 is the [B][H0][W0][C0] map after the
+ *      patch-embedding stem; stage_out is a HOST array of num_stages device pointers receiving each stage's final
+ *      map [B][Hs][Ws][Cs].  Ratio arrays are HOST arrays with one entry per block pair. ---- */
+size_t       mixaq_backbone_workspace_bytes(const mixaq_backbone_params* p, int B, int H0, int W0);
+mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params* p, const float* x0,
+                                    float* const* stage_out, int B, int H0, int W0,
+                                    const float* low_ratio_per_pair, const float* prune_ratio_per_pair /* nullable */,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Number of kernel launches the last block / merge / backbone call of this context issued. */
+int          mixaq_last_launch_count(const mixaq_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXAQ_H */

@@ -1,0 +1,345 @@
+"""Thin Python binding of the C ABI in include/mixaq.h (ctypes).  Argument marshalling only: every step of
+the path runs in the library's kernels.  PyTorch supplies device memory and the CUDA stream, nothing else.
+There is no fallback: if libmixaq.so is missing or no CUDA device is present, calls raise."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from types import SimpleNamespace
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmixaq.so")
+_lib = None
+
+EXPORTS = [
+    "mixaq_create", "mixaq_destroy", "mixaq_last_error", "mixaq_last_device_status", "mixaq_low_count",
+    "mixaq_branch_counts", "mixaq_block_prepared_bytes", "mixaq_block_prepare", "mixaq_merge_prepared_bytes",
+    "mixaq_merge_prepare", "mixaq_stage_energy", "mixaq_block_workspace_bytes", "mixaq_block_forward",
+    "mixaq_merge_workspace_bytes", "mixaq_merge_forward", "mixaq_backbone_workspace_bytes",
+    "mixaq_backbone_forward", "mixaq_last_launch_count",
+]
+
+STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
+          -5: "DEVICE_TIMEOUT", -6: "INTERNAL"}
+
+
+class MixaqError(RuntimeError):
+    def __init__(self, status, msg=""):
+        super().__init__(f"mixaq: {STATUS.get(status, status)} {msg}")
+        self.status = status
+
+
+class AQ(C.Structure):
+    _fields_ = [("bits", C.c_int), ("scale", C.c_float), ("inv_scale", C.c_float), ("zero_point", C.c_int)]
+
+
+class LinearS(C.Structure):
+    _fields_ = [("codes", C.c_void_p), ("scale", C.c_void_p), ("out_features", C.c_int), ("in_features", C.c_int),
+                ("bits", C.c_int)]
+
+
+class BranchS(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln1_g", "ln1_b", "ln2_g", "ln2_b", "b_qkv", "b_proj", "b_fc1", "b_fc2")] + \
+               [(n, AQ) for n in ("qkv_in", "q", "k", "v", "proj_in", "fc1_in", "fc2_in")] + [("bits", C.c_int)]
+
+
+class BlockS(C.Structure):
+    _fields_ = [("dim", C.c_int), ("heads", C.c_int), ("window", C.c_int), ("shift", C.c_int), ("hidden", C.c_int),
+                ("qkv", LinearS), ("proj", LinearS), ("fc1", LinearS), ("fc2", LinearS),
+                ("relpos_table", C.c_void_p), ("hi", BranchS), ("lo", BranchS),
+                ("score_inv_scale", C.c_float), ("prepared", C.c_void_p)]
+
+
+class MergeS(C.Structure):
+    _fields_ = [("ln_g", C.c_void_p), ("ln_b", C.c_void_p), ("in_", AQ), ("reduction", LinearS),
+                ("prepared", C.c_void_p)]
+
+
+class SelectOpts(C.Structure):
+    _fields_ = [("energy", C.c_void_p), ("reverse", C.c_int)]
+
+
+class Selection(C.Structure):
+    _fields_ = [("cls", C.c_void_p), ("order", C.c_void_p), ("score", C.c_void_p)]
+
+
+_TAP_FIELDS = ("a_codes", "qkv_acc", "qkv_codes", "p_codes", "pv_acc", "o_codes", "proj_acc", "x1",
+               "f1_codes", "fc1_acc", "f2_codes", "fc2_acc")
+
+
+class BranchTaps(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _TAP_FIELDS]
+
+
+class Taps(C.Structure):
+    _fields_ = [("hi", BranchTaps), ("lo", BranchTaps)]
+
+
+class BackboneS(C.Structure):
+    _fields_ = [("num_stages", C.c_int), ("depths", C.POINTER(C.c_int)), ("blocks", C.POINTER(BlockS)),
+                ("merges", C.POINTER(MergeS))]
+
+
+def lib():
+    """Loads libmixaq.so.  Raises if it has not been built: the product has no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise MixaqError(-4, f"{LIB_PATH} is missing: build it with paper_2507_19131_b200/build.py")
+        L = C.CDLL(LIB_PATH)
+        L.mixaq_last_error.restype = C.c_char_p
+        for n in ("mixaq_block_prepared_bytes", "mixaq_merge_prepared_bytes", "mixaq_block_workspace_bytes",
+                  "mixaq_merge_workspace_bytes", "mixaq_backbone_workspace_bytes"):
+            getattr(L, n).restype = C.c_size_t
+        L.mixaq_low_count.argtypes = [C.c_float, C.c_int]
+        _lib = L
+    return _lib
+
+
+def low_count(ratio: float, n: int) -> int:
+    return lib().mixaq_low_count(C.c_float(ratio), n)
+
+
+def branch_counts(H: int, W: int, low_ratio: float, prune_ratio: float = 0.0, window: int = 7):
+    cnt = (C.c_int * 3)()
+    st = lib().mixaq_branch_counts(H, W, window, C.c_float(low_ratio), C.c_float(prune_ratio), cnt)
+    if st != 0:
+        raise MixaqError(st)
+    return tuple(cnt)
+
+
+def _stream_ptr() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class Context:
+    """One library context per device (mixaq_create / mixaq_destroy)."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise MixaqError(-4, "no CUDA device: the library has no CPU path")
+        self.device = torch.device("cuda", device)
+        torch.cuda.set_device(self.device)
+        self.h = C.c_void_p()
+        st = lib().mixaq_create(C.byref(self.h), device)
+        if st != 0:
+            raise MixaqError(st, "mixaq_create")
+
+    def check(self, st: int, what: str = ""):
+        if st != 0:
+            raise MixaqError(st, what + ": " + lib().mixaq_last_error(self.h).decode())
+
+    def device_status(self) -> int:
+        return lib().mixaq_last_device_status(self.h, _stream_ptr())
+
+    def launch_count(self) -> int:
+        return lib().mixaq_last_launch_count(self.h)
+
+    def close(self):
+        if self.h:
+            lib().mixaq_destroy(self.h)
+            self.h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _aq(q) -> AQ:
+    return AQ(int(q.bits), float(q.scale), float(q.inv_scale), int(q.zp))
+
+
+class _Dev:
+    """Uploads numpy parameters once and keeps the device tensors alive."""
+
+    def __init__(self, device):
+        self.device = device
+        self.keep = []
+
+    def up(self, a: np.ndarray, dtype) -> C.c_void_p:
+        t = torch.from_numpy(np.ascontiguousarray(a, dtype=dtype)).to(self.device)
+        self.keep.append(t)
+        return C.c_void_p(t.data_ptr())
+
+    def empty(self, nbytes: int) -> C.c_void_p:
+        t = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=self.device)
+        self.keep.append(t)
+        return C.c_void_p(t.data_ptr())
+
+
+def _linear(dev: _Dev, L) -> LinearS:
+    return LinearS(dev.up(L.codes, np.int8), dev.up(L.scale, np.float32), L.codes.shape[0], L.codes.shape[1], int(L.bits))
+
+
+def _branch(dev: _Dev, b, cache) -> BranchS:
+    s = BranchS()
+    for n in ("ln1_g", "ln1_b", "ln2_g", "ln2_b", "b_qkv", "b_proj", "b_fc1", "b_fc2"):
+        a = getattr(b, n)
+        if id(a) not in cache:          # shared biases are uploaded once and aliased
+            cache[id(a)] = dev.up(a, np.float32)
+        setattr(s, n, cache[id(a)])
+    for n in ("qkv_in", "q", "k", "v", "proj_in", "fc1_in", "fc2_in"):
+        setattr(s, n, _aq(getattr(b, n)))
+    s.bits = int(b.bits)
+    return s
+
+
+def fill_block_struct(dev: _Dev, blk) -> BlockS:
+    s = BlockS()
+    s.dim, s.heads, s.window, s.shift, s.hidden = blk.dim, blk.heads, blk.window, blk.shift, blk.hidden
+    s.qkv, s.proj, s.fc1, s.fc2 = (_linear(dev, getattr(blk, n)) for n in ("qkv", "proj", "fc1", "fc2"))
+    s.relpos_table = dev.up(blk.relpos, np.float32)
+    cache = {}
+    s.hi, s.lo = _branch(dev, blk.hi, cache), _branch(dev, blk.lo, cache)
+    s.score_inv_scale = float(blk.score_inv_scale)
+    s.prepared = dev.empty(lib().mixaq_block_prepared_bytes(C.byref(s)))
+    return s
+
+
+def fill_merge_struct(dev: _Dev, m) -> MergeS:
+    s = MergeS(dev.up(m.ln_g, np.float32), dev.up(m.ln_b, np.float32), _aq(m.aq), _linear(dev, m.red), None)
+    s.prepared = dev.empty(lib().mixaq_merge_prepared_bytes(C.byref(s)))
+    return s
+
+
+class DeviceBlock:
+    """Parameters of one Two-Branch Swin Block resident on the device, prepared (mixaq_block_prepare)."""
+
+    def __init__(self, ctx: Context, blk):
+        self.ctx, self.blk = ctx, blk
+        self.dev = _Dev(ctx.device)
+        self.s = fill_block_struct(self.dev, blk)
+        ctx.check(lib().mixaq_block_prepare(ctx.h, C.byref(self.s), _stream_ptr()), "block_prepare")
+        self._ws = None
+
+    def workspace(self, B, H, W) -> torch.Tensor:
+        need = lib().mixaq_block_workspace_bytes(C.byref(self.s), B, H, W)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.ctx.device)
+        return self._ws
+
+
+def stage_energy(ctx: Context, x: torch.Tensor, score_inv_scale: float) -> torch.Tensor:
+    B, H, W, Cc = x.shape
+    e = torch.empty((B, H, W), dtype=torch.int32, device=x.device)
+    ctx.check(lib().mixaq_stage_energy(ctx.h, _ptr(x), _ptr(e), B, H, W, Cc, C.c_float(score_inv_scale), _stream_ptr()),
+              "stage_energy")
+    return e
+
+
+def _alloc_taps(device, M, slots, Cc, hidden, heads, bits):
+    u8, i32, f32 = torch.uint8, torch.int32, torch.float32
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
+    t = SimpleNamespace(
+        a_codes=z((M, Cc * bits // 8), u8), qkv_acc=z((M, 3 * Cc), i32), qkv_codes=z((M, 3 * Cc * bits // 8), u8),
+        p_codes=z((slots, heads, 49, 49), u8), pv_acc=z((M, Cc), i32), o_codes=z((M, Cc * bits // 8), u8),
+        proj_acc=z((M, Cc), i32), x1=z((M, Cc), f32), f1_codes=z((M, Cc * bits // 8), u8),
+        fc1_acc=z((M, hidden), i32), f2_codes=z((M, hidden * bits // 8), u8), fc2_acc=z((M, Cc), i32))
+    s = BranchTaps()
+    for n in _TAP_FIELDS:
+        setattr(s, n, _ptr(getattr(t, n)))
+    return t, s
+
+
+def block_forward(ctx: Context, db: DeviceBlock, x: torch.Tensor, low_ratio: float, prune_ratio: float = 0.0,
+                  energy: Optional[torch.Tensor] = None, reverse: bool = False, selection: bool = False,
+                  taps: bool = False, y: Optional[torch.Tensor] = None):
+    """mixaq_block_forward.  x: [B,H,W,C] float32 CUDA tensor.  Returns a namespace with y (and, on request,
+    cls / order / scores / counts and the per-branch taps)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    B, H, W, Cc = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    ws = db.workspace(B, H, W)
+    out = SimpleNamespace(y=y, counts=branch_counts(H, W, low_ratio, prune_ratio))
+    nW = -(-H // 7) * -(-W // 7)
+    opts = SelectOpts(_ptr(energy), 1 if reverse else 0)
+    sel = None
+    if selection:
+        out.cls = torch.empty((B, nW), dtype=torch.uint8, device=x.device)
+        out.order = torch.empty((B, nW), dtype=torch.int32, device=x.device)
+        out.scores = torch.empty((B, nW), dtype=torch.int64, device=x.device)
+        sel = Selection(_ptr(out.cls), _ptr(out.order), _ptr(out.scores))
+    tp = None
+    if taps:
+        n_hi, n_lo, _ = out.counts
+        out.hi, th = _alloc_taps(x.device, B * n_hi * 49, B * n_hi, Cc, db.blk.hidden, db.blk.heads, db.blk.hi.bits)
+        out.lo, tl = _alloc_taps(x.device, B * n_lo * 49, B * n_lo, Cc, db.blk.hidden, db.blk.heads, db.blk.lo.bits)
+        tp = Taps(th, tl)
+    st = lib().mixaq_block_forward(ctx.h, C.byref(db.s), _ptr(x), _ptr(y), B, H, W, C.c_float(low_ratio),
+                                   C.c_float(prune_ratio), C.byref(opts), C.byref(sel) if sel is not None else None,
+                                   _ptr(ws), C.c_size_t(ws.numel()), C.byref(tp) if tp is not None else None,
+                                   _stream_ptr())
+    ctx.check(st, "block_forward")
+    return out
+
+
+class DeviceMerge:
+    def __init__(self, ctx: Context, m):
+        self.ctx, self.m = ctx, m
+        self.dev = _Dev(ctx.device)
+        self.s = fill_merge_struct(self.dev, m)
+        ctx.check(lib().mixaq_merge_prepare(ctx.h, C.byref(self.s), _stream_ptr()), "merge_prepare")
+
+
+def merge_forward(ctx: Context, dm: DeviceMerge, x: torch.Tensor) -> torch.Tensor:
+    B, H, W, Cc = x.shape
+    y = torch.empty((B, (H + 1) // 2, (W + 1) // 2, 2 * Cc), dtype=torch.float32, device=x.device)
+    need = lib().mixaq_merge_workspace_bytes(C.byref(dm.s), B, H, W)
+    ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+    ctx.check(lib().mixaq_merge_forward(ctx.h, C.byref(dm.s), _ptr(x), _ptr(y), B, H, W, _ptr(ws), C.c_size_t(need),
+                                        _stream_ptr()), "merge_forward")
+    return y
+
+
+class DeviceBackbone:
+    """All parameters of a backbone on the device, prepared; owns the workspace and the stage outputs."""
+
+    def __init__(self, ctx: Context, bb, B: int, H0: int, W0: int):
+        self.ctx, self.bb, self.B, self.H0, self.W0 = ctx, bb, B, H0, W0
+        self.dev = _Dev(ctx.device)
+        nb = len(bb.blocks)
+        self.blocks = (BlockS * nb)(*[fill_block_struct(self.dev, b) for b in bb.blocks])
+        self.merges = (MergeS * max(1, len(bb.merges)))(*[fill_merge_struct(self.dev, m) for m in bb.merges])
+        self.depths = (C.c_int * len(bb.depths))(*bb.depths)
+        self.s = BackboneS(len(bb.depths), self.depths, self.blocks, self.merges)
+        for i in range(nb):
+            ctx.check(lib().mixaq_block_prepare(ctx.h, C.byref(self.blocks[i]), _stream_ptr()), "block_prepare")
+        for i in range(len(bb.merges)):
+            ctx.check(lib().mixaq_merge_prepare(ctx.h, C.byref(self.merges[i]), _stream_ptr()), "merge_prepare")
+        need = lib().mixaq_backbone_workspace_bytes(C.byref(self.s), B, H0, W0)
+        if need == 0:
+            raise MixaqError(-1, "backbone_workspace_bytes returned 0")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=ctx.device)
+        self.outs, h, w = [], H0, W0
+        for s, c in enumerate(bb.dims):
+            if s > 0:
+                h, w = (h + 1) // 2, (w + 1) // 2
+            self.outs.append(torch.empty((B, h, w, c), dtype=torch.float32, device=ctx.device))
+        self.out_ptrs = (C.c_void_p * len(self.outs))(*[o.data_ptr() for o in self.outs])
+        self.npairs = (nb + 1) // 2
+
+
+def backbone_forward(ctx: Context, dbb: DeviceBackbone, x0: torch.Tensor, low_ratios: Sequence[float],
+                     prune_ratios: Optional[Sequence[float]] = None) -> List[torch.Tensor]:
+    """mixaq_backbone_forward.  Returns the per-stage output tensors owned by `dbb` (overwritten by the next call)."""
+    assert x0.is_cuda and x0.dtype == torch.float32 and x0.is_contiguous()
+    assert tuple(x0.shape[:3]) == (dbb.B, dbb.H0, dbb.W0)
+    lr = (C.c_float * dbb.npairs)(*[float(r) for r in low_ratios][:dbb.npairs])
+    pr = None
+    if prune_ratios is not None:
+        pr = (C.c_float * dbb.npairs)(*[float(r) for r in prune_ratios][:dbb.npairs])
+    st = lib().mixaq_backbone_forward(ctx.h, C.byref(dbb.s), _ptr(x0), dbb.out_ptrs, dbb.B, dbb.H0, dbb.W0, lr, pr,
+                                      _ptr(dbb.ws), C.c_size_t(dbb.ws.numel()), _stream_ptr())
+    ctx.check(st, "backbone_forward")
+    return dbb.outs

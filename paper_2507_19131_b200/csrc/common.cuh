@@ -1,0 +1,169 @@
+// Device-side building blocks of the numeric contract shared by all kernels of the library:
+// every binary32 value that feeds a quantizer is produced by individually rounded IEEE operations in a
+// fixed order, so that integer codes do not depend on compiler contraction or on the launch shape.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mixaq {
+
+constexpr int WS = 7;         // window side
+constexpr int WT = 49;        // tokens per window
+constexpr int HEAD_DIM = 32;
+
+struct AQ {                   // activation quantizer in kernel-friendly form
+  float scale, inv_scale, zpf, qmaxf;
+  int zp, bits;
+};
+
+__device__ __forceinline__ float magic_round_add() { return 12582912.0f; }   // 1.5 * 2^23
+
+// 2^t by a round-to-nearest split t = n + f and a degree-5 polynomial in f (Horner, fused multiply-adds);
+// n goes straight into the exponent field.  Valid for t in [-125, 127].
+__device__ __forceinline__ float exp2_core(float t) {
+  const float M = 12582912.0f;
+  float r = __fadd_rn(t, M);
+  float nf = __fsub_rn(r, M);
+  float f = __fsub_rn(t, nf);
+  float p = __uint_as_float(0x3aafc47du);
+  p = __fmaf_rn(p, f, __uint_as_float(0x3c1e883du));
+  p = __fmaf_rn(p, f, __uint_as_float(0x3d635716u));
+  p = __fmaf_rn(p, f, __uint_as_float(0x3e75fc83u));
+  p = __fmaf_rn(p, f, __uint_as_float(0x3f317219u));
+  p = __fmaf_rn(p, f, __uint_as_float(0x3f800001u));
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(r) << 23));
+}
+
+// GELU(v) = max(v,0) - a*Phi(-a), a = min(|v|, 5); log2 Phi(-a) is a degree-7 polynomial on [0,5].
+__device__ __forceinline__ float gelu_f(float v) {
+  float a = fminf(fabsf(v), 5.0f);
+  float q = __uint_as_float(0xb5d6f9e3u);
+  q = __fmaf_rn(q, a, __uint_as_float(0x38729e20u));
+  q = __fmaf_rn(q, a, __uint_as_float(0xba6dcc74u));
+  q = __fmaf_rn(q, a, __uint_as_float(0x3c0a3aedu));
+  q = __fmaf_rn(q, a, __uint_as_float(0xbd5c93e3u));
+  q = __fmaf_rn(q, a, __uint_as_float(0xbeeac5d4u));
+  q = __fmaf_rn(q, a, __uint_as_float(0xbf935b8fu));
+  q = __fmaf_rn(q, a, __uint_as_float(0xbf7fffbeu));
+  float h = __fmul_rn(a, exp2_core(q));
+  return __fsub_rn(fmaxf(v, 0.0f), h);
+}
+
+// q = clamp(rne(x*inv_scale) + zp, 0, qmax)
+__device__ __forceinline__ uint32_t quant_code(float x, const AQ& q) {
+  float t = __fmul_rn(x, q.inv_scale);
+  float r = rintf(t);
+  float c = __fadd_rn(r, q.zpf);
+  c = fminf(fmaxf(c, 0.0f), q.qmaxf);
+  return (uint32_t)__float2int_rz(c);
+}
+
+// Sum over a warp by the butterfly of the contract (offsets 16, 8, 4, 2, 1); every lane ends with the
+// same bits because binary32 addition is commutative.
+__device__ __forceinline__ float warp_sum_butterfly(float v) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, off));
+  return v;
+}
+
+// LayerNorm statistics of one row held as NPL values per lane (lane l holds channels l, l+32, ...).
+template <int NPL>
+__device__ __forceinline__ void ln_stats(const float (&x)[NPL], float fC, float& mean, float& rstd) {
+  float s = 0.0f;
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) s = __fadd_rn(s, x[i]);
+  mean = __fdiv_rn(warp_sum_butterfly(s), fC);
+  float v = 0.0f;
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) { float d = __fsub_rn(x[i], mean); v = __fmaf_rn(d, d, v); }
+  float var = __fdiv_rn(warp_sum_butterfly(v), fC);
+  rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, 1e-5f)));
+}
+
+__device__ __forceinline__ float ln_apply(float x, float mean, float rstd, float g, float b) {
+  return __fmaf_rn(__fmul_rn(__fsub_rn(x, mean), rstd), g, b);
+}
+
+// Store the codes of one row that a warp holds in the lane-strided layout (lane l: channels l + 32*i).
+// bits = 8: one byte per code.  bits = 4 / 2: neighbouring lanes are merged into bytes, little end first.
+template <int NPL>
+__device__ __forceinline__ void store_codes_lane_strided(uint8_t* row, const uint32_t (&code)[NPL], int bits, int lane) {
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) {
+    uint32_t c = code[i];
+    if (bits == 8) {
+      row[lane + 32 * i] = (uint8_t)c;
+    } else if (bits == 4) {
+      uint32_t hi = __shfl_down_sync(0xffffffffu, c, 1);
+      if ((lane & 1) == 0) row[(lane + 32 * i) >> 1] = (uint8_t)(c | (hi << 4));
+    } else {  // 2 bits
+      uint32_t c1 = __shfl_down_sync(0xffffffffu, c, 1);
+      uint32_t c2 = __shfl_down_sync(0xffffffffu, c, 2);
+      uint32_t c3 = __shfl_down_sync(0xffffffffu, c, 3);
+      if ((lane & 3) == 0) row[(lane + 32 * i) >> 2] = (uint8_t)(c | (c1 << 2) | (c2 << 4) | (c3 << 6));
+    }
+  }
+}
+
+// 32 consecutive codes of one row (held by ONE thread) packed and stored with vector stores.
+// dst points at the first byte of the group; it is 32*bits/8-byte aligned by construction.
+__device__ __forceinline__ void store_codes_32(uint8_t* dst, const uint32_t (&c)[32], int bits) {
+  if (bits == 8) {
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = c[4 * i] | (c[4 * i + 1] << 8) | (c[4 * i + 2] << 16) | (c[4 * i + 3] << 24);
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  } else if (bits == 4) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v |= c[8 * i + e] << (4 * e);
+      w[i] = v;
+    }
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+  } else {
+    uint32_t w[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) v |= c[16 * i + e] << (2 * e);
+      w[i] = v;
+    }
+    reinterpret_cast<uint2*>(dst)[0] = make_uint2(w[0], w[1]);
+  }
+}
+
+// Unpack 32 consecutive codes (one k-group) from packed storage into 32 bytes (eight 32-bit words).
+__device__ __forceinline__ void load_codes_32(const uint8_t* src, int bits, uint32_t (&w)[8]) {
+  if (bits == 8) {
+    uint4 a = reinterpret_cast<const uint4*>(src)[0], b = reinterpret_cast<const uint4*>(src)[1];
+    w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+  } else if (bits == 4) {
+    uint4 a = reinterpret_cast<const uint4*>(src)[0];
+    uint32_t p[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {   // 8 nibbles -> 8 bytes
+      uint32_t v = p[i];
+      uint32_t lo = (v & 0xFu) | ((v & 0xF0u) << 4) | ((v & 0xF00u) << 8) | ((v & 0xF000u) << 12);
+      v >>= 16;
+      uint32_t hi = (v & 0xFu) | ((v & 0xF0u) << 4) | ((v & 0xF00u) << 8) | ((v & 0xF000u) << 12);
+      w[2 * i] = lo; w[2 * i + 1] = hi;
+    }
+  } else {
+    uint2 a = reinterpret_cast<const uint2*>(src)[0];
+    uint32_t p[2] = {a.x, a.y};
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {   // one byte of 4 codes -> 4 bytes
+        uint32_t v = (p[i] >> (8 * j)) & 0xFFu;
+        w[4 * i + j] = (v & 0x3u) | ((v & 0xCu) << 6) | ((v & 0x30u) << 12) | ((v & 0xC0u) << 18);
+      }
+  }
+}
+
+}  // namespace mixaq

@@ -1,0 +1,94 @@
+// Internal interface between the host API (mixaq.cu) and the kernel translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "common.cuh"
+
+namespace mixaq {
+
+extern int g_launches;   // kernels launched since the API call started (host bookkeeping)
+
+// ---- selection ------------------------------------------------------------------------------
+void launch_energy(const float* x, int32_t* energy, long ntok, int C, float inv_scale, cudaStream_t st);
+
+struct SelectArgs {
+  const int32_t* energy;     // [B][H][W]
+  int64_t* score;            // [B][nW]
+  int32_t* order;            // [B][nW]
+  uint8_t* cls;              // [B][nW]
+  int32_t* rowsrc_hi;        // [B*n_hi*49] source token (b*H*W + y*W + x) or -1 for a pad token
+  int32_t* rowsrc_lo;        // [B*n_lo*49]
+  int32_t* rowsrc_pr;        // [B*n_pr*49]
+  int32_t* win_hi;           // [B*n_hi] window index of every batch slot
+  int32_t* win_lo;           // [B*n_lo]
+  int B, H, W, shift, nwx, nW, n_hi, n_lo, n_pr, reverse;
+};
+void launch_select(const SelectArgs& a, cudaStream_t st);   // 2 launches
+
+// ---- row-wise LayerNorm + quantize + pack -----------------------------------------------------
+struct LnBranch {
+  const float* src;          // feature map (gather) or window-batch matrix [M][C]
+  const int32_t* rowsrc;     // nullable: row m reads src + rowsrc[m]*C (rowsrc < 0: pad token -> zero after LN)
+  const float *gamma, *beta;
+  uint8_t* out;              // [M][C*bits/8]
+  AQ q;
+  int M;
+};
+void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st);
+
+struct MergeGatherArgs {
+  const float* x; const float *gamma, *beta; uint8_t* out; AQ q; int B, H, W, C;
+};
+void launch_merge_gather(const MergeGatherArgs& a, cudaStream_t st);
+void launch_copy_rows(const float* x, float* y, const int32_t* rowsrc, int M, int C, cudaStream_t st);
+
+// ---- integer GEMM with fused epilogues ----------------------------------------------------------
+enum EpiMode { EPI_QKV = 0, EPI_PROJ = 1, EPI_FC1 = 2, EPI_FC2 = 3, EPI_MERGE = 4 };
+
+struct GemmBranch {
+  const uint8_t* a;          // [M][K*a_bits/8] packed unsigned codes
+  int M, a_bits;
+  const float* mult;         // [N]  s_a * s_w[n]
+  const int32_t* zc;         // [N]  z_a * sum_k w[n][k]
+  const float* bias;         // [N]  (nullable for EPI_MERGE)
+  AQ q0, q1, q2;             // output quantizers (QKV: q,k,v; FC1: q0)
+  int out_bits;
+  uint8_t* out_codes;        // QKV, FC1: [M][N*out_bits/8]
+  float* out_f;              // PROJ: x1 [M][N];  FC2: y feature map;  MERGE: [M][N]
+  const float* res;          // PROJ: feature map x (gathered through rowsrc);  FC2: x1 [M][N]
+  const int32_t* rowsrc;     // PROJ, FC2
+  int32_t* tap_acc;          // nullable [M][N]
+};
+struct GemmArgs {
+  const int8_t* w;           // [N][K]
+  int N, K, C;               // C: channels per q/k/v section (EPI_QKV)
+  int mode;
+  GemmBranch br[2];
+};
+void launch_gemm(const GemmArgs& g, cudaStream_t st);
+
+// ---- fused window attention ----------------------------------------------------------------------
+struct AttnBranch {
+  const uint8_t* qkv;        // [M][3C*bits/8]
+  uint8_t* out;              // [M][C*bits/8]
+  const int32_t* win;        // [slots] window index (for the shift mask)
+  AQ q, k, v, o;
+  int bits, slots;
+  float alpha;               // s_q*s_k/sqrt(d)
+  float so;                  // s_p*s_v
+  uint8_t* tap_p;            // nullable
+  int32_t* tap_pv;           // nullable
+};
+struct AttnArgs {
+  const float* relbias;      // [heads][49][49]
+  int C, heads, shift, Hp, Wp, nwx, nW;
+  AttnBranch br[2];
+};
+void launch_attention(const AttnArgs& a, cudaStream_t st);
+
+// ---- preparation -----------------------------------------------------------------------------------
+void launch_prepare_linear(const int8_t* w, const float* sw, int N, int K, float sa, int za, float* mult,
+                           int32_t* zc, cudaStream_t st);
+void launch_prepare_relbias(const float* table, int heads, float* out, cudaStream_t st);
+
+}  // namespace mixaq

@@ -1,0 +1,509 @@
+// Host side of the C ABI declared in include/mixaq.h: argument validation, workspace carving, the launch
+// schedule of one Two-Branch Swin Block (MixA-Q Section 3.2, Figure 3) and of the backbone loop.
+// Nothing here computes: every step of the path runs in the kernels.
+#include "../../include/mixaq.h"
+#include "kernels.h"
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+namespace mixaq {
+bool ln_dim_supported(int C);
+bool merge_dim_supported(int C);
+void launch_gemm_simple(const GemmArgs& g, cudaStream_t st);
+int g_launches = 0;
+}  // namespace mixaq
+
+using namespace mixaq;
+
+struct mixaq_ctx {
+  int device;
+  int* d_status;
+  int launches;
+  char err[256];
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct Carver {
+  char* base; size_t off;
+  explicit Carver(void* p) : base((char*)p), off(0) {}
+  template <class T> T* take(size_t n) { T* p = base ? (T*)(base + off) : nullptr; off += align_up(n * sizeof(T)); return p; }
+};
+
+AQ to_aq(const mixaq_aq& q) {
+  AQ a; a.scale = q.scale; a.inv_scale = q.inv_scale; a.zp = q.zero_point; a.bits = q.bits;
+  a.zpf = (float)q.zero_point; a.qmaxf = (float)((1 << q.bits) - 1);
+  return a;
+}
+
+mixaq_status fail(mixaq_ctx* ctx, mixaq_status s, const char* msg) {
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
+  return s;
+}
+
+mixaq_status check_cuda(mixaq_ctx* ctx, const char* where) {
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return MIXAQ_OK;
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s: %s", where, cudaGetErrorString(e));
+  return MIXAQ_CUDA_ERROR;
+}
+
+bool bits_ok(int b) { return b == 8 || b == 4 || b == 2; }
+bool aq_ok(const mixaq_aq& q, int bits) {
+  return q.bits == bits && q.scale > 0.f && q.inv_scale > 0.f && q.zero_point >= 0 && q.zero_point < (1 << bits);
+}
+bool linear_ok(const mixaq_linear& l, int out_f, int in_f) {
+  return l.codes && l.scale && l.out_features == out_f && l.in_features == in_f;
+}
+bool branch_ok(const mixaq_branch& b) {
+  if (!bits_ok(b.bits)) return false;
+  if (!b.ln1_g || !b.ln1_b || !b.ln2_g || !b.ln2_b || !b.b_qkv || !b.b_proj || !b.b_fc1 || !b.b_fc2) return false;
+  return aq_ok(b.qkv_in, b.bits) && aq_ok(b.q, b.bits) && aq_ok(b.k, b.bits) && aq_ok(b.v, b.bits) &&
+         aq_ok(b.proj_in, b.bits) && aq_ok(b.fc1_in, b.bits) && aq_ok(b.fc2_in, b.bits);
+}
+
+mixaq_status validate_block(mixaq_ctx* ctx, const mixaq_block_params* p) {
+  if (!p) return fail(ctx, MIXAQ_INVALID_ARG, "block params are NULL");
+  if (p->window != WS) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "window must be 7");
+  if (p->dim <= 0 || p->dim % 32 || !ln_dim_supported(p->dim)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "unsupported dim");
+  if (p->heads <= 0 || p->dim != p->heads * HEAD_DIM) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "dim/heads must be 32");
+  if (p->hidden <= 0 || p->hidden % 32) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "hidden must be a multiple of 32");
+  if (p->shift < 0 || p->shift >= WS) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "shift must be in [0, window)");
+  if (!linear_ok(p->qkv, 3 * p->dim, p->dim) || !linear_ok(p->proj, p->dim, p->dim) ||
+      !linear_ok(p->fc1, p->hidden, p->dim) || !linear_ok(p->fc2, p->dim, p->hidden))
+    return fail(ctx, MIXAQ_INVALID_ARG, "weight matrix missing or of the wrong shape");
+  if (!p->relpos_table) return fail(ctx, MIXAQ_INVALID_ARG, "relpos_table is NULL");
+  if (!branch_ok(p->hi) || !branch_ok(p->lo)) return fail(ctx, MIXAQ_INVALID_ARG, "branch parameters invalid");
+  if (!(p->score_inv_scale > 0.f)) return fail(ctx, MIXAQ_INVALID_ARG, "score_inv_scale must be positive");
+  return MIXAQ_OK;
+}
+
+// layout of a block's prepared buffer
+struct Prepared {
+  float* mult[4][2]; int32_t* zc[4][2]; float* relbias; size_t bytes;
+};
+Prepared carve_prepared(const mixaq_block_params* p, void* base) {
+  Prepared r; Carver c(base);
+  const int N[4] = {3 * p->dim, p->dim, p->hidden, p->dim};
+  for (int l = 0; l < 4; ++l)
+    for (int b = 0; b < 2; ++b) { r.mult[l][b] = c.take<float>(N[l]); r.zc[l][b] = c.take<int32_t>(N[l]); }
+  r.relbias = c.take<float>((size_t)p->heads * WT * WT);
+  r.bytes = c.off;
+  return r;
+}
+
+struct Geometry { int Hp, Wp, nwx, nW, n_hi, n_lo, n_pr; };
+Geometry geometry(int H, int W, float low, float prune) {
+  Geometry g;
+  g.Hp = (H + WS - 1) / WS * WS; g.Wp = (W + WS - 1) / WS * WS;
+  g.nwx = g.Wp / WS; g.nW = (g.Hp / WS) * g.nwx;
+  g.n_pr = mixaq_low_count(prune, g.nW);
+  g.n_lo = mixaq_low_count(low, g.nW - g.n_pr);
+  g.n_hi = g.nW - g.n_pr - g.n_lo;
+  return g;
+}
+
+// workspace of one block call; sized for the worst split (all windows in the wider branch)
+struct BlockWs {
+  int32_t* energy; int64_t* score; int32_t* order; uint8_t* cls;
+  int32_t *rowsrc[3], *win[2];
+  uint8_t *a[2], *qkv[2], *o[2], *f1[2], *f2[2]; float* x1[2];
+  size_t bytes;
+};
+BlockWs carve_block(const mixaq_block_params* p, int B, int H, int W, void* base) {
+  BlockWs w; Carver c(base);
+  Geometry g = geometry(H, W, 0.f, 0.f);
+  const size_t slots = (size_t)B * g.nW, rows = slots * WT;
+  const int C = p->dim, Hd = p->hidden;
+  w.energy = c.take<int32_t>((size_t)B * H * W);
+  w.score = c.take<int64_t>(slots); w.order = c.take<int32_t>(slots); w.cls = c.take<uint8_t>(slots);
+  for (int i = 0; i < 3; ++i) w.rowsrc[i] = c.take<int32_t>(rows);
+  for (int i = 0; i < 2; ++i) w.win[i] = c.take<int32_t>(slots);
+  for (int i = 0; i < 2; ++i) {
+    const int bits = i == 0 ? p->hi.bits : p->lo.bits;
+    w.a[i]   = c.take<uint8_t>(rows * C * bits / 8);
+    w.qkv[i] = c.take<uint8_t>(rows * 3 * C * bits / 8);
+    w.o[i]   = c.take<uint8_t>(rows * C * bits / 8);
+    w.x1[i]  = c.take<float>(rows * C);
+    w.f1[i]  = c.take<uint8_t>(rows * C * bits / 8);
+    w.f2[i]  = c.take<uint8_t>(rows * Hd * bits / 8);
+  }
+  w.bytes = c.off;
+  return w;
+}
+
+void fill_gemm_branch(GemmBranch& g, const uint8_t* a, int M, int a_bits, const float* mult, const int32_t* zc,
+                      const float* bias) {
+  memset(&g, 0, sizeof(g));
+  g.a = a; g.M = M; g.a_bits = a_bits; g.mult = mult; g.zc = zc; g.bias = bias;
+}
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+int mixaq_low_count(float ratio, int n) { return (int)std::floor((double)ratio * (double)n + 1e-6); }
+
+mixaq_status mixaq_branch_counts(int H, int W, int window, float low_ratio, float prune_ratio, int* counts) {
+  if (!counts || window != WS || H <= 0 || W <= 0) return MIXAQ_INVALID_ARG;
+  if (!(low_ratio >= 0.f && low_ratio <= 1.f) || !(prune_ratio >= 0.f && prune_ratio <= 1.f)) return MIXAQ_INVALID_ARG;
+  Geometry g = geometry(H, W, low_ratio, prune_ratio);
+  counts[0] = g.n_hi; counts[1] = g.n_lo; counts[2] = g.n_pr;
+  return MIXAQ_OK;
+}
+
+mixaq_status mixaq_create(mixaq_ctx** out, int device) {
+  if (!out) return MIXAQ_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
+  if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
+  mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
+  if (!c) return MIXAQ_INTERNAL;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr;
+  if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError(); delete c; return MIXAQ_CUDA_ERROR;
+  }
+  *out = c;
+  return MIXAQ_OK;
+}
+
+mixaq_status mixaq_destroy(mixaq_ctx* ctx) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+  return MIXAQ_OK;
+}
+
+const char* mixaq_last_error(const mixaq_ctx* ctx) { return ctx ? ctx->err : "no context"; }
+int mixaq_last_launch_count(const mixaq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  int h = 0;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaMemcpyAsync(&h, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return check_cuda(ctx, "status read") == MIXAQ_OK ? MIXAQ_CUDA_ERROR : MIXAQ_CUDA_ERROR;
+  return h == 0 ? MIXAQ_OK : MIXAQ_DEVICE_TIMEOUT;
+}
+
+// -------------------------------------------------------------------------------------------------
+size_t mixaq_block_prepared_bytes(const mixaq_block_params* p) {
+  if (!p || p->dim <= 0 || p->hidden <= 0 || p->heads <= 0) return 0;
+  return carve_prepared(p, nullptr).bytes;
+}
+
+mixaq_status mixaq_block_prepare(mixaq_ctx* ctx, const mixaq_block_params* p, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  mixaq_status s = validate_block(ctx, p);
+  if (s != MIXAQ_OK) return s;
+  if (!p->prepared) return fail(ctx, MIXAQ_INVALID_ARG, "prepared buffer is NULL");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Prepared pr = carve_prepared(p, p->prepared);
+  const mixaq_linear* L[4] = {&p->qkv, &p->proj, &p->fc1, &p->fc2};
+  for (int b = 0; b < 2; ++b) {
+    const mixaq_branch& br = b == 0 ? p->hi : p->lo;
+    const mixaq_aq* in[4] = {&br.qkv_in, &br.proj_in, &br.fc1_in, &br.fc2_in};
+    for (int l = 0; l < 4; ++l)
+      launch_prepare_linear(L[l]->codes, L[l]->scale, L[l]->out_features, L[l]->in_features, in[l]->scale,
+                            in[l]->zero_point, pr.mult[l][b], pr.zc[l][b], st);
+  }
+  launch_prepare_relbias(p->relpos_table, p->heads, pr.relbias, st);
+  return check_cuda(ctx, "block_prepare");
+}
+
+size_t mixaq_merge_prepared_bytes(const mixaq_merge_params* p) {
+  if (!p || p->reduction.out_features <= 0) return 0;
+  return align_up((size_t)p->reduction.out_features * 4) * 2;
+}
+
+mixaq_status mixaq_merge_prepare(mixaq_ctx* ctx, const mixaq_merge_params* p, void* cuda_stream) {
+  if (!ctx || !p) return MIXAQ_INVALID_ARG;
+  if (!p->prepared || !p->reduction.codes || !p->reduction.scale) return fail(ctx, MIXAQ_INVALID_ARG, "merge params incomplete");
+  Carver c(p->prepared);
+  float* mult = c.take<float>(p->reduction.out_features);
+  int32_t* zc = c.take<int32_t>(p->reduction.out_features);
+  launch_prepare_linear(p->reduction.codes, p->reduction.scale, p->reduction.out_features, p->reduction.in_features,
+                        p->in.scale, p->in.zero_point, mult, zc, (cudaStream_t)cuda_stream);
+  return check_cuda(ctx, "merge_prepare");
+}
+
+mixaq_status mixaq_stage_energy(mixaq_ctx* ctx, const float* x, int32_t* energy, int B, int H, int W, int C,
+                                float score_inv_scale, void* cuda_stream) {
+  if (!ctx || !x || !energy || B <= 0 || H <= 0 || W <= 0 || C <= 0 || !(score_inv_scale > 0.f)) return MIXAQ_INVALID_ARG;
+  launch_energy(x, energy, (long)B * H * W, C, score_inv_scale, (cudaStream_t)cuda_stream);
+  return check_cuda(ctx, "stage_energy");
+}
+
+// -------------------------------------------------------------------------------------------------
+size_t mixaq_block_workspace_bytes(const mixaq_block_params* p, int B, int H, int W) {
+  if (!p || B <= 0 || H <= 0 || W <= 0 || p->dim <= 0 || p->hidden <= 0) return 0;
+  return carve_block(p, B, H, W, nullptr).bytes;
+}
+
+mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, const float* x, float* y,
+                                 int B, int H, int W, float low_ratio, float prune_ratio,
+                                 const mixaq_select_opts* opts, const mixaq_selection* sel_out,
+                                 void* workspace, size_t workspace_bytes, const mixaq_taps* taps,
+                                 void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  mixaq_status s = validate_block(ctx, p);
+  if (s != MIXAQ_OK) return s;
+  if (!x || !y || x == y) return fail(ctx, MIXAQ_INVALID_ARG, "x / y NULL or aliased");
+  if (B <= 0 || H <= 0 || W <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "B, H, W must be positive");
+  if (!(low_ratio >= 0.f && low_ratio <= 1.f) || !(prune_ratio >= 0.f && prune_ratio <= 1.f))
+    return fail(ctx, MIXAQ_INVALID_ARG, "ratios must lie in [0, 1]");
+  if (!p->prepared) return fail(ctx, MIXAQ_INVALID_ARG, "block was not prepared (prepared == NULL)");
+  if ((long)B * H * W >= (1L << 31) / WT) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many tokens");
+  Geometry g = geometry(H, W, low_ratio, prune_ratio);
+  if ((size_t)g.nW * 8 > 48 * 1024) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many windows per image (max 6144)");
+  if (!workspace) return fail(ctx, MIXAQ_INVALID_ARG, "workspace is NULL");
+  BlockWs ws = carve_block(p, B, H, W, workspace);
+  if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "workspace too small");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int C = p->dim, Hd = p->hidden;
+  Prepared pr = carve_prepared(p, p->prepared);
+  g_launches = 0;
+
+  // 1. scores and selection
+  const int32_t* energy = opts ? opts->energy : nullptr;
+  if (!energy) { launch_energy(x, ws.energy, (long)B * H * W, C, p->score_inv_scale, st); energy = ws.energy; }
+  SelectArgs sa;
+  sa.energy = energy; sa.score = ws.score; sa.order = ws.order; sa.cls = ws.cls;
+  sa.rowsrc_hi = ws.rowsrc[0]; sa.rowsrc_lo = ws.rowsrc[1]; sa.rowsrc_pr = ws.rowsrc[2];
+  sa.win_hi = ws.win[0]; sa.win_lo = ws.win[1];
+  sa.B = B; sa.H = H; sa.W = W; sa.shift = p->shift; sa.nwx = g.nwx; sa.nW = g.nW;
+  sa.n_hi = g.n_hi; sa.n_lo = g.n_lo; sa.n_pr = g.n_pr; sa.reverse = opts ? opts->reverse : 0;
+  launch_select(sa, st);
+  if (sel_out) {
+    const size_t n = (size_t)B * g.nW;
+    if (sel_out->cls)   cudaMemcpyAsync(sel_out->cls, ws.cls, n, cudaMemcpyDeviceToDevice, st);
+    if (sel_out->order) cudaMemcpyAsync(sel_out->order, ws.order, n * 4, cudaMemcpyDeviceToDevice, st);
+    if (sel_out->score) cudaMemcpyAsync(sel_out->score, ws.score, n * 8, cudaMemcpyDeviceToDevice, st);
+  }
+
+  const mixaq_branch* brp[2] = {&p->hi, &p->lo};
+  const int M[2] = {B * g.n_hi * WT, B * g.n_lo * WT};
+  const int slots[2] = {B * g.n_hi, B * g.n_lo};
+  const mixaq_branch_taps* tp[2] = {taps ? &taps->hi : nullptr, taps ? &taps->lo : nullptr};
+
+  // 2. gather + LN1 + quantize + pack
+  LnBranch lb[2];
+  for (int i = 0; i < 2; ++i) {
+    lb[i].src = x; lb[i].rowsrc = ws.rowsrc[i]; lb[i].gamma = brp[i]->ln1_g; lb[i].beta = brp[i]->ln1_b;
+    lb[i].out = ws.a[i]; lb[i].q = to_aq(brp[i]->qkv_in); lb[i].M = M[i];
+  }
+  launch_ln_quant(lb[0], lb[1], C, st);
+
+  // 3. QKV GEMM -> q, k, v codes
+  GemmArgs ga;
+  ga.w = p->qkv.codes; ga.N = 3 * C; ga.K = C; ga.C = C; ga.mode = EPI_QKV;
+  for (int i = 0; i < 2; ++i) {
+    fill_gemm_branch(ga.br[i], ws.a[i], M[i], brp[i]->bits, pr.mult[0][i], pr.zc[0][i], brp[i]->b_qkv);
+    ga.br[i].q0 = to_aq(brp[i]->q); ga.br[i].q1 = to_aq(brp[i]->k); ga.br[i].q2 = to_aq(brp[i]->v);
+    ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.qkv[i];
+    ga.br[i].tap_acc = tp[i] ? tp[i]->qkv_acc : nullptr;
+  }
+  launch_gemm(ga, st);
+
+  // 4. window attention
+  AttnArgs aa;
+  aa.relbias = pr.relbias; aa.C = C; aa.heads = p->heads; aa.shift = p->shift; aa.Hp = g.Hp; aa.Wp = g.Wp;
+  aa.nwx = g.nwx; aa.nW = g.nW;
+  const float rs = (float)(1.0 / std::sqrt((double)HEAD_DIM));
+  for (int i = 0; i < 2; ++i) {
+    AttnBranch& ab = aa.br[i];
+    ab.qkv = ws.qkv[i]; ab.out = ws.o[i]; ab.win = ws.win[i];
+    ab.q = to_aq(brp[i]->q); ab.k = to_aq(brp[i]->k); ab.v = to_aq(brp[i]->v); ab.o = to_aq(brp[i]->proj_in);
+    ab.bits = brp[i]->bits; ab.slots = slots[i];
+    ab.alpha = (brp[i]->q.scale * brp[i]->k.scale) * rs;
+    ab.so = (1.0f / (float)((1 << brp[i]->bits) - 1)) * brp[i]->v.scale;
+    ab.tap_p = tp[i] ? tp[i]->p_codes : nullptr; ab.tap_pv = tp[i] ? tp[i]->pv_acc : nullptr;
+  }
+  launch_attention(aa, st);
+
+  // 5. proj GEMM + attention residual -> x1
+  ga.w = p->proj.codes; ga.N = C; ga.K = C; ga.mode = EPI_PROJ;
+  for (int i = 0; i < 2; ++i) {
+    fill_gemm_branch(ga.br[i], ws.o[i], M[i], brp[i]->bits, pr.mult[1][i], pr.zc[1][i], brp[i]->b_proj);
+    ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = ws.rowsrc[i];
+    ga.br[i].tap_acc = tp[i] ? tp[i]->proj_acc : nullptr;
+  }
+  launch_gemm(ga, st);
+
+  // 6. LN2 + quantize + pack
+  for (int i = 0; i < 2; ++i) {
+    lb[i].src = ws.x1[i]; lb[i].rowsrc = nullptr; lb[i].gamma = brp[i]->ln2_g; lb[i].beta = brp[i]->ln2_b;
+    lb[i].out = ws.f1[i]; lb[i].q = to_aq(brp[i]->fc1_in); lb[i].M = M[i];
+  }
+  launch_ln_quant(lb[0], lb[1], C, st);
+
+  // 7. fc1 GEMM + GELU + requantize
+  ga.w = p->fc1.codes; ga.N = Hd; ga.K = C; ga.mode = EPI_FC1;
+  for (int i = 0; i < 2; ++i) {
+    fill_gemm_branch(ga.br[i], ws.f1[i], M[i], brp[i]->bits, pr.mult[2][i], pr.zc[2][i], brp[i]->b_fc1);
+    ga.br[i].q0 = to_aq(brp[i]->fc2_in); ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.f2[i];
+    ga.br[i].tap_acc = tp[i] ? tp[i]->fc1_acc : nullptr;
+  }
+  launch_gemm(ga, st);
+
+  // 8. fc2 GEMM + residual + scatter (reverse shift, crop)
+  ga.w = p->fc2.codes; ga.N = C; ga.K = Hd; ga.mode = EPI_FC2;
+  for (int i = 0; i < 2; ++i) {
+    fill_gemm_branch(ga.br[i], ws.f2[i], M[i], brp[i]->bits, pr.mult[3][i], pr.zc[3][i], brp[i]->b_fc2);
+    ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = ws.rowsrc[i];
+    ga.br[i].tap_acc = tp[i] ? tp[i]->fc2_acc : nullptr;
+  }
+  launch_gemm(ga, st);
+
+  // 9. pruned windows are forwarded unchanged
+  launch_copy_rows(x, y, ws.rowsrc[2], B * g.n_pr * WT, C, st);
+
+  if (taps) {
+    for (int i = 0; i < 2; ++i) {
+      const size_t rows = (size_t)M[i]; const int bits = brp[i]->bits;
+      if (rows == 0) continue;
+      if (tp[i]->a_codes)   cudaMemcpyAsync(tp[i]->a_codes, ws.a[i], rows * C * bits / 8, cudaMemcpyDeviceToDevice, st);
+      if (tp[i]->qkv_codes) cudaMemcpyAsync(tp[i]->qkv_codes, ws.qkv[i], rows * 3 * C * bits / 8, cudaMemcpyDeviceToDevice, st);
+      if (tp[i]->o_codes)   cudaMemcpyAsync(tp[i]->o_codes, ws.o[i], rows * C * bits / 8, cudaMemcpyDeviceToDevice, st);
+      if (tp[i]->x1)        cudaMemcpyAsync(tp[i]->x1, ws.x1[i], rows * C * 4, cudaMemcpyDeviceToDevice, st);
+      if (tp[i]->f1_codes)  cudaMemcpyAsync(tp[i]->f1_codes, ws.f1[i], rows * C * bits / 8, cudaMemcpyDeviceToDevice, st);
+      if (tp[i]->f2_codes)  cudaMemcpyAsync(tp[i]->f2_codes, ws.f2[i], rows * Hd * bits / 8, cudaMemcpyDeviceToDevice, st);
+    }
+  }
+  ctx->launches = g_launches;
+  return check_cuda(ctx, "block_forward");
+}
+
+// -------------------------------------------------------------------------------------------------
+size_t mixaq_merge_workspace_bytes(const mixaq_merge_params* p, int B, int H, int W) {
+  if (!p || B <= 0 || H <= 0 || W <= 0) return 0;
+  const size_t toks = (size_t)B * ((H + 1) / 2) * ((W + 1) / 2);
+  return align_up(toks * p->reduction.in_features * p->in.bits / 8);
+}
+
+mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
+                                 int B, int H, int W, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !p) return MIXAQ_INVALID_ARG;
+  if (!x || !y || !workspace || B <= 0 || H <= 0 || W <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "merge: bad argument");
+  const int K = p->reduction.in_features, N = p->reduction.out_features, C = K / 4;
+  if (K % 4 || N % 32 || !merge_dim_supported(C)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "merge: unsupported dims");
+  if (!p->ln_g || !p->ln_b || !p->reduction.codes || !p->reduction.scale || !p->prepared || !bits_ok(p->in.bits) ||
+      !aq_ok(p->in, p->in.bits))
+    return fail(ctx, MIXAQ_INVALID_ARG, "merge params incomplete");
+  if (mixaq_merge_workspace_bytes(p, B, H, W) > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "merge workspace");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  g_launches = 0;
+  const int M = B * ((H + 1) / 2) * ((W + 1) / 2);
+  MergeGatherArgs mg;
+  mg.x = x; mg.gamma = p->ln_g; mg.beta = p->ln_b; mg.out = (uint8_t*)workspace; mg.q = to_aq(p->in);
+  mg.B = B; mg.H = H; mg.W = W; mg.C = C;
+  launch_merge_gather(mg, st);
+  Carver c(p->prepared);
+  float* mult = c.take<float>(N);
+  int32_t* zc = c.take<int32_t>(N);
+  GemmArgs ga;
+  ga.w = p->reduction.codes; ga.N = N; ga.K = K; ga.C = N; ga.mode = EPI_MERGE;
+  fill_gemm_branch(ga.br[0], (const uint8_t*)workspace, M, p->in.bits, mult, zc, nullptr);
+  ga.br[0].out_f = y;
+  fill_gemm_branch(ga.br[1], nullptr, 0, p->in.bits, mult, zc, nullptr);
+  launch_gemm(ga, st);
+  ctx->launches = g_launches;
+  return check_cuda(ctx, "merge_forward");
+}
+
+// -------------------------------------------------------------------------------------------------
+namespace {
+struct BackboneWs { float* scratch; int32_t* energy; void* merge; void* block; size_t merge_bytes, block_bytes, bytes; };
+BackboneWs carve_backbone(const mixaq_backbone_params* p, int B, int H0, int W0, void* base) {
+  BackboneWs w; Carver c(base);
+  size_t max_map = 0, max_tok = 0, max_merge = 0, max_block = 0;
+  int H = H0, W = W0, blk = 0;
+  for (int s = 0; s < p->num_stages; ++s) {
+    if (s > 0) {
+      max_merge = std::max(max_merge, mixaq_merge_workspace_bytes(&p->merges[s - 1], B, H, W));
+      H = (H + 1) / 2; W = (W + 1) / 2;
+    }
+    const mixaq_block_params* b0 = &p->blocks[blk];
+    max_map = std::max(max_map, (size_t)B * H * W * b0->dim);
+    max_tok = std::max(max_tok, (size_t)B * H * W);
+    for (int i = 0; i < p->depths[s]; ++i, ++blk)
+      max_block = std::max(max_block, mixaq_block_workspace_bytes(&p->blocks[blk], B, H, W));
+  }
+  w.scratch = c.take<float>(max_map);
+  w.energy = c.take<int32_t>(max_tok);
+  w.merge = c.take<uint8_t>(max_merge); w.merge_bytes = align_up(max_merge);
+  w.block = c.take<uint8_t>(max_block); w.block_bytes = align_up(max_block);
+  w.bytes = c.off;
+  return w;
+}
+}  // namespace
+
+size_t mixaq_backbone_workspace_bytes(const mixaq_backbone_params* p, int B, int H0, int W0) {
+  if (!p || !p->depths || !p->blocks || p->num_stages <= 0 || B <= 0 || H0 <= 0 || W0 <= 0) return 0;
+  if (p->num_stages > 1 && !p->merges) return 0;
+  return carve_backbone(p, B, H0, W0, nullptr).bytes;
+}
+
+mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params* p, const float* x0,
+                                    float* const* stage_out, int B, int H0, int W0,
+                                    const float* low_ratio_per_pair, const float* prune_ratio_per_pair,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  if (!p || !p->depths || !p->blocks || p->num_stages <= 0 || (p->num_stages > 1 && !p->merges))
+    return fail(ctx, MIXAQ_INVALID_ARG, "backbone params incomplete");
+  if (!x0 || !stage_out || !low_ratio_per_pair || !workspace || B <= 0 || H0 <= 0 || W0 <= 0)
+    return fail(ctx, MIXAQ_INVALID_ARG, "backbone: bad argument");
+  int nblk = 0;
+  for (int s = 0; s < p->num_stages; ++s) {
+    if (p->depths[s] <= 0 || (p->depths[s] != 1 && p->depths[s] % 2)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "depths must be even or 1");
+    if (!stage_out[s]) return fail(ctx, MIXAQ_INVALID_ARG, "stage_out entry is NULL");
+    nblk += p->depths[s];
+  }
+  for (int b = 0; b < nblk; ++b) {
+    mixaq_status s = validate_block(ctx, &p->blocks[b]);
+    if (s != MIXAQ_OK) return s;
+    float r = low_ratio_per_pair[b / 2], q = prune_ratio_per_pair ? prune_ratio_per_pair[b / 2] : 0.f;
+    if (!(r >= 0.f && r <= 1.f) || !(q >= 0.f && q <= 1.f)) return fail(ctx, MIXAQ_INVALID_ARG, "ratios must lie in [0, 1]");
+  }
+  BackboneWs ws = carve_backbone(p, B, H0, W0, workspace);
+  if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "backbone workspace too small");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int total = 0, H = H0, W = W0, blk = 0;
+  const float* cur = x0;
+  for (int s = 0; s < p->num_stages; ++s) {
+    const int d = p->depths[s];
+    float* out_s = stage_out[s];
+    if (s > 0) {
+      // the merge writes where the first block of the stage does NOT write
+      float* mdst = (d % 2 == 0) ? out_s : ws.scratch;
+      mixaq_status r = mixaq_merge_forward(ctx, &p->merges[s - 1], cur, mdst, B, H, W, ws.merge, ws.merge_bytes, st);
+      if (r != MIXAQ_OK) return r;
+      total += ctx->launches;
+      cur = mdst; H = (H + 1) / 2; W = (W + 1) / 2;
+    }
+    const mixaq_block_params* b0 = &p->blocks[blk];
+    launch_energy(cur, ws.energy, (long)B * H * W, b0->dim, b0->score_inv_scale, st);
+    total += 1;
+    mixaq_select_opts so; so.energy = ws.energy; so.reverse = 0;
+    for (int i = 0; i < d; ++i, ++blk) {
+      float* dst = ((d - 1 - i) % 2 == 0) ? out_s : ws.scratch;
+      mixaq_status r = mixaq_block_forward(ctx, &p->blocks[blk], cur, dst, B, H, W, low_ratio_per_pair[blk / 2],
+                                           prune_ratio_per_pair ? prune_ratio_per_pair[blk / 2] : 0.f, &so, nullptr,
+                                           ws.block, ws.block_bytes, nullptr, st);
+      if (r != MIXAQ_OK) return r;
+      total += ctx->launches;
+      cur = dst;
+    }
+  }
+  ctx->launches = total;
+  return check_cuda(ctx, "backbone_forward");
+}
+
+}  // extern "C"

@@ -1,0 +1,130 @@
+// Memory-bound row kernels: gather + LayerNorm + quantize + bit-pack (both branches in one launch),
+// the patch-merging gather, and the pass-through copy of pruned windows (MixA-Q Section 3.2 / 3.4).
+// One warp owns one token row; lane l holds channels l, l+32, l+64, ... so every load is a full 128-byte line.
+#include "kernels.h"
+
+namespace mixaq {
+
+template <int NPL>
+__global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo) {
+  const int C = NPL * 32;
+  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  int lane = threadIdx.x & 31;
+  if (row >= hi.M + lo.M) return;
+  const bool is_hi = row < hi.M;
+  const LnBranch& br = is_hi ? hi : lo;
+  int m = is_hi ? row : row - hi.M;
+  long srow = m;
+  if (br.rowsrc) srow = br.rowsrc[m];
+  uint32_t code[NPL];
+  if (srow < 0) {
+    // pad token: zero after the normalisation, i.e. the code of 0.0
+    AQ q = br.q;
+    uint32_t z = quant_code(0.0f, q);
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) code[i] = z;
+  } else {
+    const float* src = br.src + srow * C;
+    float x[NPL];
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) x[i] = __ldg(src + lane + 32 * i);
+    float mean, rstd;
+    ln_stats<NPL>(x, (float)C, mean, rstd);
+    AQ q = br.q;
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) {
+      int c = lane + 32 * i;
+      code[i] = quant_code(ln_apply(x[i], mean, rstd, __ldg(br.gamma + c), __ldg(br.beta + c)), q);
+    }
+  }
+  int bits = br.q.bits;
+  store_codes_lane_strided<NPL>(br.out + (long)m * (C * bits / 8), code, bits, lane);
+}
+
+// patch merging: token (b, y2, x2) of the output gathers (2y2+dy, 2x2+dx) for (dy,dx) = (0,0),(1,0),(0,1),(1,1)
+// in this order along the channel axis; neighbours outside the map are zeros (they do take part in the LN).
+template <int NPL>   // NPL = 4C/32
+__global__ void __launch_bounds__(256) k_merge_gather(MergeGatherArgs a) {
+  const int K = NPL * 32;
+  const int C = K / 4;
+  int H2 = (a.H + 1) / 2, W2 = (a.W + 1) / 2;
+  long tok = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  int lane = threadIdx.x & 31;
+  if (tok >= (long)a.B * H2 * W2) return;
+  int b = (int)(tok / ((long)H2 * W2));
+  int r = (int)(tok - (long)b * H2 * W2);
+  int y2 = r / W2, x2 = r - y2 * W2;
+  float x[NPL];
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) {
+    int c = lane + 32 * i;
+    int g = c / C, cc = c - g * C;
+    int yy = 2 * y2 + (g & 1), xx = 2 * x2 + (g >> 1);
+    x[i] = (yy < a.H && xx < a.W) ? __ldg(a.x + (((long)b * a.H + yy) * a.W + xx) * C + cc) : 0.0f;
+  }
+  float mean, rstd;
+  ln_stats<NPL>(x, (float)K, mean, rstd);
+  uint32_t code[NPL];
+  AQ q = a.q;
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) {
+    int c = lane + 32 * i;
+    code[i] = quant_code(ln_apply(x[i], mean, rstd, __ldg(a.gamma + c), __ldg(a.beta + c)), q);
+  }
+  store_codes_lane_strided<NPL>(a.out + tok * (K * q.bits / 8), code, q.bits, lane);
+}
+
+__global__ void __launch_bounds__(256) k_copy_rows(const float* __restrict__ x, float* __restrict__ y,
+                                                   const int32_t* __restrict__ rowsrc, int M, int C) {
+  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  long s = rowsrc[row];
+  if (s < 0) return;
+  for (int c = lane; c < C; c += 32) y[s * C + c] = __ldg(x + s * C + c);
+}
+
+#define MIXAQ_NPL_CASE(n, KERNEL, ...) case n: KERNEL<n><<<grid, 256, 0, st>>>(__VA_ARGS__); break;
+
+void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st) {
+  int rows = hi.M + lo.M;
+  if (rows == 0) return;
+  unsigned grid = (rows + 7) / 8;
+  switch (C / 32) {
+    MIXAQ_NPL_CASE(1, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(2, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(3, k_ln_quant, hi, lo)
+    MIXAQ_NPL_CASE(4, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(6, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(8, k_ln_quant, hi, lo)
+    MIXAQ_NPL_CASE(12, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(16, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(24, k_ln_quant, hi, lo)
+    MIXAQ_NPL_CASE(32, k_ln_quant, hi, lo)
+    default: return;   // rejected by the host API before any launch
+  }
+  ++g_launches;
+}
+
+void launch_merge_gather(const MergeGatherArgs& a, cudaStream_t st) {
+  long toks = (long)a.B * ((a.H + 1) / 2) * ((a.W + 1) / 2);
+  unsigned grid = (unsigned)((toks + 7) / 8);
+  switch (4 * a.C / 32) {
+    MIXAQ_NPL_CASE(4, k_merge_gather, a) MIXAQ_NPL_CASE(8, k_merge_gather, a) MIXAQ_NPL_CASE(12, k_merge_gather, a)
+    MIXAQ_NPL_CASE(16, k_merge_gather, a) MIXAQ_NPL_CASE(24, k_merge_gather, a) MIXAQ_NPL_CASE(32, k_merge_gather, a)
+    MIXAQ_NPL_CASE(48, k_merge_gather, a) MIXAQ_NPL_CASE(64, k_merge_gather, a)
+    default: return;
+  }
+  ++g_launches;
+}
+
+void launch_copy_rows(const float* x, float* y, const int32_t* rowsrc, int M, int C, cudaStream_t st) {
+  if (M == 0) return;
+  k_copy_rows<<<(M + 7) / 8, 256, 0, st>>>(x, y, rowsrc, M, C);
+  ++g_launches;
+}
+
+bool ln_dim_supported(int C) {
+  switch (C / 32) { case 1: case 2: case 3: case 4: case 6: case 8: case 12: case 16: case 24: case 32: return C % 32 == 0; }
+  return false;
+}
+bool merge_dim_supported(int C) {
+  switch (4 * C / 32) { case 4: case 8: case 12: case 16: case 24: case 32: case 48: case 64: return C % 32 == 0; }
+  return false;
+}
+
+}  // namespace mixaq

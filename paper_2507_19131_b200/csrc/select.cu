@@ -1,0 +1,96 @@
+// Window importance scoring and ratio-driven selection (MixA-Q Section 3.2; pruned class: Section 3.4).
+// Integer work throughout: int8 score codes, int32 token energies, int64 window scores, ranks by counting.
+#include "kernels.h"
+
+namespace mixaq {
+
+// One warp per token: energy = sum_c clamp(rne(x*inv), -127, 127)^2.
+__global__ void __launch_bounds__(256) k_energy(const float* __restrict__ x, int32_t* __restrict__ energy,
+                                                long ntok, int C, float inv) {
+  long tok = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  int lane = threadIdx.x & 31;
+  if (tok >= ntok) return;
+  const float* row = x + tok * C;
+  int e = 0;
+  for (int c = lane; c < C; c += 32) {
+    float r = rintf(__fmul_rn(__ldg(row + c), inv));
+    r = fminf(fmaxf(r, -127.0f), 127.0f);
+    int code = __float2int_rz(r);
+    e += code * code;
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) e += __shfl_xor_sync(0xffffffffu, e, off);
+  if (lane == 0) energy[tok] = e;
+}
+
+__device__ __forceinline__ int window_src(int b, int H, int W, int Hp, int Wp, int shift, int nwx, int w, int t) {
+  int wy = w / nwx, wx = w - wy * nwx;
+  int i = t / WS, j = t - i * WS;
+  int y = wy * WS + i + shift; if (y >= Hp) y -= Hp;
+  int x = wx * WS + j + shift; if (x >= Wp) x -= Wp;
+  if (y >= H || x >= W) return -1;
+  return (b * H + y) * W + x;
+}
+
+// One warp per (image, window): score = sum of the energies of the window's real tokens under this
+// block's own (possibly shifted, cyclically wrapped) partition.
+__global__ void __launch_bounds__(256) k_window_score(SelectArgs a) {
+  int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  int lane = threadIdx.x & 31;
+  if (gw >= a.B * a.nW) return;
+  int b = gw / a.nW, w = gw - b * a.nW;
+  int Hp = (a.H + WS - 1) / WS * WS, Wp = (a.W + WS - 1) / WS * WS;
+  long long s = 0;
+  for (int t = lane; t < WT; t += 32) {
+    int src = window_src(b, a.H, a.W, Hp, Wp, a.shift, a.nwx, w, t);
+    if (src >= 0) s += a.energy[src];
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+  if (lane == 0) a.score[gw] = s;
+}
+
+// Rank by counting: rank(w) = #{v : v precedes w in (score desc, index asc)}; ranks are a permutation.
+// The thread that owns window w also writes the batch bookkeeping of its slot.
+__global__ void __launch_bounds__(128) k_rank_emit(SelectArgs a) {
+  extern __shared__ long long s_score[];
+  int b = blockIdx.y;
+  const int64_t* sc = a.score + (long)b * a.nW;
+  for (int i = threadIdx.x; i < a.nW; i += blockDim.x) s_score[i] = sc[i];
+  __syncthreads();
+  int w = blockIdx.x * blockDim.x + threadIdx.x;
+  if (w >= a.nW) return;
+  long long mine = s_score[w];
+  int rank = 0;
+  if (!a.reverse) {
+    for (int v = 0; v < a.nW; ++v) { long long o = s_score[v]; rank += (o > mine) || (o == mine && v < w); }
+  } else {
+    for (int v = 0; v < a.nW; ++v) { long long o = s_score[v]; rank += (o < mine) || (o == mine && v < w); }
+  }
+  a.order[(long)b * a.nW + rank] = w;
+  int c = rank < a.n_hi ? 0 : (rank < a.n_hi + a.n_lo ? 1 : 2);
+  a.cls[(long)b * a.nW + w] = (uint8_t)c;
+  int Hp = (a.H + WS - 1) / WS * WS, Wp = (a.W + WS - 1) / WS * WS;
+  int32_t* dst; long slot;
+  if (c == 0)      { slot = (long)b * a.n_hi + rank;                   dst = a.rowsrc_hi; a.win_hi[slot] = w; }
+  else if (c == 1) { slot = (long)b * a.n_lo + (rank - a.n_hi);        dst = a.rowsrc_lo; a.win_lo[slot] = w; }
+  else             { slot = (long)b * a.n_pr + (rank - a.n_hi - a.n_lo); dst = a.rowsrc_pr; }
+  for (int t = 0; t < WT; ++t) dst[slot * WT + t] = window_src(b, a.H, a.W, Hp, Wp, a.shift, a.nwx, w, t);
+}
+
+void launch_energy(const float* x, int32_t* energy, long ntok, int C, float inv_scale, cudaStream_t st) {
+  int wpb = 8;
+  k_energy<<<(unsigned)((ntok + wpb - 1) / wpb), wpb * 32, 0, st>>>(x, energy, ntok, C, inv_scale);
+  ++g_launches;
+}
+
+void launch_select(const SelectArgs& a, cudaStream_t st) {
+  int nwin = a.B * a.nW;
+  k_window_score<<<(nwin + 7) / 8, 256, 0, st>>>(a);
+  ++g_launches;
+  dim3 grid((a.nW + 127) / 128, a.B);
+  k_rank_emit<<<grid, 128, (size_t)a.nW * sizeof(long long), st>>>(a);
+  ++g_launches;
+}
+
+}  // namespace mixaq

@@ -1,0 +1,188 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle on the same seeded inputs.
+Integer results (scores, selection, packed codes, zero-point-corrected int32 accumulators) must be bit-exact;
+binary32 results must agree within 1e-3 of the output's max magnitude (they are expected to be identical)."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from paper_2507_19131_b200 import synth  # noqa: E402
+
+F32 = np.float32
+TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def mq():
+    from paper_2507_19131_b200 import binding
+    if not torch.cuda.is_available():
+        pytest.fail("GPU test selected but no CUDA device is visible")
+    return binding
+
+
+@pytest.fixture(scope="module")
+def ctx(mq):
+    c = mq.Context(0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def dev(x):
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def assert_close_rel(got, want, tol=TOL):
+    scale = max(float(np.abs(want).max()), 1e-30)
+    err = float(np.abs(got.astype(np.float64) - want.astype(np.float64)).max())
+    assert err <= tol * scale, f"max abs err {err} > {tol} * {scale}"
+
+
+def check_taps(orc, blk, ref, got, counts):
+    """Every intermediate of both branches, bit for bit."""
+    for name, br, n in (("hi", blk.hi, counts[0]), ("lo", blk.lo, counts[1])):
+        r, g = getattr(ref, name), getattr(got, name)
+        if n == 0:
+            continue
+        bits = br.bits
+        for f in ("a_codes", "qkv_codes", "o_codes", "f1_codes", "f2_codes"):
+            assert np.array_equal(g.__dict__[f].cpu().numpy(), orc.pack(r.__dict__[f], bits)), f"{name}.{f}"
+        for f in ("qkv_acc", "pv_acc", "proj_acc", "fc1_acc", "fc2_acc", "p_codes"):
+            assert np.array_equal(g.__dict__[f].cpu().numpy(), r.__dict__[f]), f"{name}.{f}"
+        assert_close_rel(g.x1.cpu().numpy(), r.x1)
+        assert np.array_equal(g.x1.cpu().numpy(), r.x1), f"{name}.x1 not bit-identical"
+
+
+def run_block_case(orc, mq, ctx, blk, x, low, prune=0.0, reverse=False, stage_energy=False, taps=True):
+    db = mq.DeviceBlock(ctx, blk)
+    xd = dev(x)
+    e_ref = e_dev = None
+    if stage_energy:
+        e_ref = orc.energy(x, blk.score_inv_scale)
+        e_dev = mq.stage_energy(ctx, xd, blk.score_inv_scale)
+        assert np.array_equal(e_dev.cpu().numpy(), e_ref)
+    ref = orc.block_forward(blk, x, low, prune, energy_map=e_ref, reverse=reverse, taps=taps)
+    got = mq.block_forward(ctx, db, xd, low, prune, energy=e_dev, reverse=reverse, selection=True, taps=taps)
+    torch.cuda.synchronize()
+    assert got.counts == ref.counts
+    assert np.array_equal(got.scores.cpu().numpy(), ref.scores)
+    assert np.array_equal(got.order.cpu().numpy(), ref.order)
+    assert np.array_equal(got.cls.cpu().numpy(), ref.cls)
+    if taps:
+        check_taps(orc, blk, ref, got, ref.counts)
+    y = got.y.cpu().numpy()
+    assert_close_rel(y, ref.y)
+    assert np.array_equal(y, ref.y), "outputs are within tolerance but not bit-identical"
+    return ref, got
+
+
+# ------------------------------------------------------------------------------------------------
+def test_selection_only_many_shapes(orc, mq, ctx):
+    rng = np.random.default_rng(0)
+    for (B, H, W, C, shift, low, prune, rev) in [(2, 16, 19, 32, 0, 0.3, 0.0, False), (2, 16, 19, 32, 3, 0.3, 0.2, False),
+                                                  (1, 56, 56, 96, 0, 0.5, 0.0, True), (3, 30, 37, 64, 3, 0.7, 0.1, False),
+                                                  (1, 7, 7, 32, 0, 0.5, 0.0, False)]:
+        blk = synth.make_block(rng, C, C // 32, shift, 8, 8, 4)
+        x = synth.input_student_t(int(rng.integers(1 << 30)), B, H, W, C)
+        x[:, : H // 2] = np.round(x[:, : H // 2])           # provoke tied scores
+        run_block_case(orc, mq, ctx, blk, x, low, prune, reverse=rev, taps=False)
+
+
+def test_all_equal_scores_break_ties_by_index(orc, mq, ctx):
+    blk = synth.make_block(np.random.default_rng(1), 32, 1, 0, 8, 8, 4)
+    x = np.ones((1, 21, 28, 32), F32)
+    ref, got = run_block_case(orc, mq, ctx, blk, x, 0.5, taps=False)
+    assert got.order.cpu().numpy()[0].tolist() == list(range(12))
+
+
+@pytest.mark.parametrize("shift", [0, 3])
+@pytest.mark.parametrize("bits", [(8, 4), (4, 2), (8, 8)])
+def test_block_tiny_all_taps(orc, mq, ctx, shift, bits):
+    blk = synth.make_block(np.random.default_rng(10 + shift), 64, 2, shift, 4, bits[0], bits[1], share_bias=False)
+    x = synth.input_blobs(11, 2, 17, 23, 64, bg_std=0.5, gain=4.0)     # ragged: padded to 21 x 28
+    run_block_case(orc, mq, ctx, blk, x, 0.4, stage_energy=bool(shift))
+
+
+def test_block_config1_all_taps(orc, mq, ctx):
+    wl = synth.config1()
+    run_block_case(orc, mq, ctx, wl.backbone.blocks[0], wl.x, 0.5)
+
+
+@pytest.mark.parametrize("low,prune", [(0.0, 0.0), (1.0, 0.0), (0.5, 0.3), (0.0, 1.0), (1.0, 0.5)])
+def test_block_degenerate_splits(orc, mq, ctx, low, prune):
+    blk = synth.make_block(np.random.default_rng(20), 32, 1, 3, 8, 8, 4)
+    x = synth.input_blobs(21, 2, 14, 22, 32, bg_std=0.5, gain=4.0)
+    ref, got = run_block_case(orc, mq, ctx, blk, x, low, prune)
+    if prune == 1.0:
+        assert np.array_equal(got.y.cpu().numpy(), x)                 # everything forwarded unchanged
+
+
+def test_block_single_window_and_wide_dims(orc, mq, ctx):
+    blk = synth.make_block(np.random.default_rng(30), 32, 1, 0, 8, 8, 4)
+    run_block_case(orc, mq, ctx, blk, synth.input_blobs(31, 1, 5, 6, 32), 0.0)
+    for dim in (128, 192, 384):
+        blk = synth.make_block(np.random.default_rng(dim), dim, dim // 32, 3, 4, 8, 4)
+        run_block_case(orc, mq, ctx, blk, synth.input_blobs(dim + 1, 1, 14, 15, dim, bg_std=0.5), 0.5)
+
+
+def test_merge_parity(orc, mq, ctx):
+    for (C, B, H, W) in [(32, 2, 9, 11), (96, 1, 20, 34), (192, 1, 13, 8)]:
+        m = synth.make_merge(np.random.default_rng(C), C, 4, 8)
+        x = synth.input_blobs(C + 5, B, H, W, C, bg_std=0.5)
+        dm = mq.DeviceMerge(ctx, m)
+        y = mq.merge_forward(ctx, dm, dev(x)).cpu().numpy()
+        want = orc.merge_forward(m, x)
+        assert_close_rel(y, want)
+        assert np.array_equal(y, want)
+
+
+@pytest.mark.parametrize("prune", [0.0, 0.2])
+def test_backbone_tiny(orc, mq, ctx, prune):
+    wl = synth.tiny_backbone(ratio=0.4, prune=prune)
+    want = orc.backbone_forward(wl.backbone, wl.x, wl.low_ratios, wl.prune_ratios)
+    dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+    got = mq.backbone_forward(ctx, dbb, dev(wl.x), wl.low_ratios, wl.prune_ratios)
+    torch.cuda.synchronize()
+    for g, w in zip(got, want):
+        assert_close_rel(g.cpu().numpy(), w)
+        assert np.array_equal(g.cpu().numpy(), w)
+
+
+def test_config2_stage1_pair_full_size(orc, mq, ctx):
+    """Block pair at 200x334 (W-MSA then SW-MSA with mask), B=2, Student-t input, ratio 0.3, shared stage energy."""
+    wl = synth.config2()
+    want = orc.backbone_forward(wl.backbone, wl.x, wl.low_ratios)
+    dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+    got = mq.backbone_forward(ctx, dbb, dev(wl.x), wl.low_ratios)
+    torch.cuda.synchronize()
+    y = got[0].cpu().numpy()
+    assert_close_rel(y, want[0])
+    assert np.array_equal(y, want[0])
+
+
+def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
+    import ctypes as C
+    blk = synth.make_block(np.random.default_rng(40), 32, 1, 0, 8, 8, 4)
+    db = mq.DeviceBlock(ctx, blk)
+    x = torch.zeros((1, 14, 14, 32), device="cuda")
+    with pytest.raises(mq.MixaqError) as e:
+        mq.block_forward(ctx, db, x, 1.5)
+    assert e.value.status == -1
+    with pytest.raises(mq.MixaqError) as e:
+        mq.block_forward(ctx, db, x, 0.5, y=x)
+    assert e.value.status == -1
+    L = mq.lib()
+    ws = db.workspace(1, 14, 14)
+    y = torch.empty_like(x)
+    st = L.mixaq_block_forward(ctx.h, C.byref(db.s), C.c_void_p(x.data_ptr()), C.c_void_p(y.data_ptr()), 1, 14, 14,
+                               C.c_float(0.5), C.c_float(0.0), None, None, C.c_void_p(ws.data_ptr()), C.c_size_t(16),
+                               None, None)
+    assert st == -3
+    bad = mq.BlockS.from_buffer_copy(db.s)
+    bad.window = 8
+    st = L.mixaq_block_forward(ctx.h, C.byref(bad), C.c_void_p(x.data_ptr()), C.c_void_p(y.data_ptr()), 1, 14, 14,
+                               C.c_float(0.5), C.c_float(0.0), None, None, C.c_void_p(ws.data_ptr()),
+                               C.c_size_t(ws.numel()), None, None)
+    assert st == -2
+    assert ctx.device_status() == 0
