@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized Two-Branch Swin backbone forward (MixA-Q) on B200.
+
+Metric: images/s of the Swin-T Two-Branch backbone at 800x1333 (200x334 tokens after the patch-4 stem),
+W4 weights, A8 high / A4 low, as a function of the low-bit ratio; the headline `value` is at --ratio.
+One "step" = one backbone forward of one synthetic image through the C ABI (mixaq_backbone_forward).
+
+  python bench.py --gpus 1 --steps 20 --warmup 3                 # this library
+  python bench.py --impl reference --steps 5 --warmup 1          # the CPU oracle, bounded sample per step
+  torchrun --nproc-per-node N bench.py --gpus N ...              # N independent replicas (weak scaling)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "swin_t_two_branch_backbone_images_per_sec_800x1333"
+UNIT = "images/s"
+SWEEP = [0.0, 0.25, 0.5, 0.75]
+L2_FLUSH_BYTES = 256 << 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.idx)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [s.strip() for s in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def workload(ratio: float):
+    from paper_2507_19131_b200 import synth
+    return synth.config3(ratio=ratio)
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work per kernel family for one backbone forward (used for the roofline of the dominant kernel)
+# ------------------------------------------------------------------------------------------------
+def algorithmic_work(wl, mq):
+    """Returns {category: dict(ops=..., bytes=...)} for ONE forward.  Window-batch rows include Swin's pad
+    tokens (the method computes them); MMA tile padding is excluded."""
+    bb = wl.backbone
+    B, H, W = wl.B, wl.H, wl.W
+    work = {}
+
+    def add(cat, ops=0.0, byt=0.0):
+        w = work.setdefault(cat, dict(ops=0.0, bytes=0.0))
+        w["ops"] += ops
+        w["bytes"] += byt
+
+    k = 0
+    for s, (C, dep) in enumerate(zip(bb.dims, bb.depths)):
+        if s > 0:
+            Cp = bb.dims[s - 1]
+            M = B * ((H + 1) // 2) * ((W + 1) // 2)
+            bits = bb.merges[s - 1].aq.bits
+            add("merge_gather_ln_quant", byt=B * H * W * Cp * 4 + M * 4 * Cp * bits / 8)
+            add("gemm_merge", ops=2.0 * M * (4 * Cp) * (2 * Cp), byt=M * 4 * Cp * bits / 8 + M * 2 * Cp * 4)
+            H, W = (H + 1) // 2, (W + 1) // 2
+        add("energy", byt=B * H * W * (C * 4 + 4))
+        for _ in range(dep):
+            blk = bb.blocks[k]
+            n_hi, n_lo, n_pr = mq.branch_counts(H, W, wl.low_ratios[k // 2], wl.prune_ratios[k // 2] if wl.prune_ratios else 0.0)
+            Hd = blk.hidden
+            for n, bits in ((n_hi, blk.hi.bits), (n_lo, blk.lo.bits)):
+                M = B * n * 49
+                cb = bits / 8.0
+                add("gather_ln1_quant", byt=M * (C * 4 + C * cb))
+                add("gemm_qkv", ops=2.0 * M * C * 3 * C, byt=M * (C * cb + 3 * C * cb))
+                add("attention", ops=2.0 * M * 2 * 49 * C, byt=M * (3 * C * cb + C * cb))
+                add("gemm_proj", ops=2.0 * M * C * C, byt=M * (C * cb + C * 4 + C * 4))
+                add("ln2_quant", byt=M * (C * 4 + C * cb))
+                add("gemm_fc1_gelu", ops=2.0 * M * C * Hd, byt=M * (C * cb + Hd * cb))
+                add("gemm_fc2_scatter", ops=2.0 * M * Hd * C, byt=M * (Hd * cb + C * 4 + C * 4))
+            add("select", byt=B * H * W * 4)
+            add("copy_pruned", byt=B * n_pr * 49 * C * 8)
+            k += 1
+    return work
+
+
+TENSOR_CATS = {"gemm_qkv", "gemm_proj", "gemm_fc1_gelu", "gemm_fc2_scatter", "gemm_merge"}
+# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None
+NCU_TRAFFIC_PER_LAUNCH = {}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2507_19131_b200 import binding as mq
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    ctx = mq.Context(local)
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def time_ratio(ratio, steps, warm, sampler=None, e2e=False):
+        wl = workload(ratio)
+        # replicas differ only in their seed-shifted input (weak scaling: one image per rank per step)
+        x_host = torch.from_numpy(np.roll(wl.x, rank, axis=1).copy()).pin_memory()
+        dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+        x_dev = x_host.cuda()
+        outs_host = [torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in dbb.outs]
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+
+        def step():
+            if e2e:
+                x_dev.copy_(x_host, non_blocking=True)
+            outs = mq.backbone_forward(ctx, dbb, x_dev, wl.low_ratios, wl.prune_ratios)
+            if e2e:
+                for h, o in zip(outs_host, outs):
+                    h.copy_(o, non_blocking=True)
+
+        for _ in range(warm):
+            step()
+        barrier()
+        if sampler:
+            sampler.start()
+        t0 = time.perf_counter()
+        for i in range(steps):
+            flush.fill_(i & 0xFF)                    # evict L2 between timed iterations (outside the events)
+            ev[i][0].record()
+            step()
+            ev[i][1].record()
+        barrier()
+        wall = time.perf_counter() - t0
+        clocks = sampler.stop() if sampler else None
+        ms = sum(a.elapsed_time(b) for a, b in ev)
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        launches = ctx.launch_count()
+        h2d = x_host.numel() * 4 if e2e else 0
+        d2h = sum(h.numel() * 4 for h in outs_host) if e2e else 0
+        return dict(ms=ms, wall=wall, clocks=clocks, launches=launches, h2d=h2d, d2h=d2h, wl=wl, dbb=dbb, x_dev=x_dev)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    main = time_ratio(args.ratio, K, Wm, sampler)
+    ms_per_step = main["ms"] / K
+    value = world * wl_images(main["wl"]) * K / (main["ms"] / 1e3)
+
+    # per-kernel CUDA-event breakdown: a separate pass of the same K steps with events around every kernel
+    ctx.profile_begin()
+    for _ in range(K):
+        mq.backbone_forward(ctx, main["dbb"], main["x_dev"], main["wl"].low_ratios, main["wl"].prune_ratios)
+    prof = ctx.profile_end()
+    work = algorithmic_work(main["wl"], mq)
+    kernels = {}
+    for cat, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        w = work.get(cat, dict(ops=0.0, bytes=0.0))
+        per_fwd_ms = ms / K
+        kernels[cat] = dict(ms_per_step=round(per_fwd_ms, 5), launches_per_step=cnt // K,
+                            share=0.0, tops=round(w["ops"] / (per_fwd_ms * 1e-3) / 1e12, 3) if w["ops"] else None,
+                            gbs=round(w["bytes"] / (per_fwd_ms * 1e-3) / 1e9, 1))
+    tot = sum(v["ms_per_step"] for v in kernels.values()) or 1.0
+    for v in kernels.values():
+        v["share"] = round(v["ms_per_step"] / tot, 4)
+    dom = max(kernels, key=lambda c: kernels[c]["ms_per_step"])
+    dk = kernels[dom]
+    if dom in TENSOR_CATS:
+        peak = 2.0 * peaks["bf16_sustained"]      # int8 dense = 2 x bf16 (nominal ratio) on the measured bf16 peak
+        roof = dict(kernel=dom, bound="tensor", achieved=dk["tops"], peak=peak, unit="TOP/s(int8)",
+                    frac=round(dk["tops"] / peak, 5),
+                    peak_source=f"2 x bf16_tflops_sustained of {peaks['source']} peaks (kernel timed inside a long step)")
+    else:
+        peak = peaks["hbm_gbs"]
+        roof = dict(kernel=dom, bound="hbm", achieved=dk["gbs"], peak=peak, unit="GB/s",
+                    frac=round(dk["gbs"] / peak, 5), peak_source=f"hbm_gbs of {peaks['source']} peaks")
+    roof["launch_us"] = round(1e3 * dk["ms_per_step"] / max(1, dk["launches_per_step"]), 3)
+    roof["traffic"] = NCU_TRAFFIC_PER_LAUNCH.get(dom)
+    roof["timed"] = "separate pass of K steps with CUDA events around every kernel, on the launching stream"
+
+    # end to end through the public call with HOST buffers (pinned): H2D of the image, forward, D2H of the 4 maps
+    e2e = time_ratio(args.ratio, K, Wm, None, e2e=True)
+    e2e_value = world * wl_images(e2e["wl"]) * K / (e2e["ms"] / 1e3)
+
+    sweep = {}
+    if args.sweep and world == 1:
+        for r in SWEEP:
+            if abs(r - args.ratio) < 1e-9:
+                sweep[str(r)] = round(value, 2)
+                continue
+            s = time_ratio(r, max(3, K // 2), 3)
+            sweep[str(r)] = round(wl_images(s["wl"]) * max(3, K // 2) / (s["ms"] / 1e3), 2)
+
+    status = ctx.device_status()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    line = {
+        "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8 MMA (int32 accumulate) + f32 epilogues", "data": "synthetic",
+        "config": {"workload": main["wl"].name, "model": "Swin-T two-branch backbone (96/192/384/768, 2/2/6/2)",
+                   "image": "800x1333", "tokens": [main["wl"].H, main["wl"].W], "batch_per_gpu": 1,
+                   "weights": "W4 (int8 container)", "act_bits_high_low": [8, 4], "low_ratio": args.ratio,
+                   "l2": f"flushed between timed iterations ({L2_FLUSH_BYTES >> 20} MiB write)",
+                   "parallelism": "replicas only (one image per GPU, no collective)"},
+        "clocks": main["clocks"],
+        "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+                "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": round(e2e["ms"] / K, 4)},
+        "gpu_launches": main["launches"] * K,
+        "roofline": roof,
+        "kernels": kernels,
+        "low_ratio_sweep_images_per_sec": sweep,
+        "device_status": status,
+    }
+    if args.cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(full=True)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def wl_images(wl):
+    return wl.B
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle as CPU baseline / reference arm
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(crop_h: int, crop_w: int, ratio: float):
+    """Times the oracle (as it stands) on a crop of the workload; returns (seconds, images-equivalent, threads)."""
+    from oracle import oracle as orc
+    wl = workload(ratio)
+    x = np.ascontiguousarray(wl.x[:, :crop_h, :crop_w])
+    t0 = time.perf_counter()
+    orc.backbone_forward(wl.backbone, x, wl.low_ratios, wl.prune_ratios)
+    dt = time.perf_counter() - t0
+    frac = (crop_h * crop_w) / float(wl.H * wl.W)
+    return dt, frac * wl.B, orc.get_threads(), wl
+
+
+def cpu_baseline(full: bool, ratio: float = 0.5):
+    if full:
+        dt, imgs, thr, wl = oracle_sample(200, 334, ratio)
+        sample = "one full forward of the same workload (1 image, 200x334 tokens)"
+    else:
+        dt, imgs, thr, wl = oracle_sample(50, 84, ratio)
+        sample = "one forward of a 50x84-token crop (6.3 % of the image's tokens), scaled by token count"
+    return {"value": round(imgs / dt, 5), "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample,
+            "seconds": round(dt, 3)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    K, Wm = args.steps, args.warmup
+    for _ in range(Wm):
+        oracle_sample(50, 84, args.ratio)
+    t0 = time.perf_counter()
+    imgs = 0.0
+    for _ in range(K):
+        dt, im, thr, wl = oracle_sample(50, 84, args.ratio)
+        imgs += im
+    total = time.perf_counter() - t0
+    value = imgs / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": K, "warmup": Wm, "ms_per_step": round(1e3 * total / K, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32/int64 integer + f32", "data": "synthetic",
+        "config": {"workload": wl.name, "low_ratio": args.ratio,
+                   "sample": "each step = one oracle forward of a 50x84-token crop (6.3 % of the tokens), scaled by token count"},
+        "cpu_baseline": {"value": round(value, 5), "unit": UNIT, "cores": thr, "kind": "oracle",
+                         "sample": "50x84-token crop per step, scaled by token count"},
+        "e2e": {"value": round(value, 5), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ratio", type=float, default=0.5)
+    ap.add_argument("--no-sweep", dest="sweep", action="store_false")
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -159,6 +159,16 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 
+/* ---- per-kernel timing (the paper reports no time breakdown; this is the library's own tracing aid).
+ *      Between begin and end every kernel family launched through this context is bracketed by CUDA events on
+ *      the launching stream.  end() synchronises the stream and returns, per category (see
+ *      mixaq_profile_category_name), the summed device milliseconds and the number of event pairs; both HOST
+ *      arrays have mixaq_profile_categories() entries.  Profiling creates events (not graph-capturable). ---- */
+int          mixaq_profile_categories(void);
+const char*  mixaq_profile_category_name(int category);
+mixaq_status mixaq_profile_begin(mixaq_ctx* ctx);
+mixaq_status mixaq_profile_end(mixaq_ctx* ctx, void* cuda_stream, float* ms_per_category, int* launches_per_category);
+
 #ifdef __cplusplus
 }
 #endif

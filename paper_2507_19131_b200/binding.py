@@ -20,7 +20,8 @@ EXPORTS = [
     "mixaq_branch_counts", "mixaq_block_prepared_bytes", "mixaq_block_prepare", "mixaq_merge_prepared_bytes",
     "mixaq_merge_prepare", "mixaq_stage_energy", "mixaq_block_workspace_bytes", "mixaq_block_forward",
     "mixaq_merge_workspace_bytes", "mixaq_merge_forward", "mixaq_backbone_workspace_bytes",
-    "mixaq_backbone_forward", "mixaq_last_launch_count",
+    "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
+    "mixaq_profile_begin", "mixaq_profile_end",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -92,6 +93,7 @@ def lib():
             raise MixaqError(-4, f"{LIB_PATH} is missing: build it with paper_2507_19131_b200/build.py")
         L = C.CDLL(LIB_PATH)
         L.mixaq_last_error.restype = C.c_char_p
+        L.mixaq_profile_category_name.restype = C.c_char_p
         for n in ("mixaq_block_prepared_bytes", "mixaq_merge_prepared_bytes", "mixaq_block_workspace_bytes",
                   "mixaq_merge_workspace_bytes", "mixaq_backbone_workspace_bytes"):
             getattr(L, n).restype = C.c_size_t
@@ -142,6 +144,16 @@ class Context:
 
     def launch_count(self) -> int:
         return lib().mixaq_last_launch_count(self.h)
+
+    def profile_begin(self):
+        self.check(lib().mixaq_profile_begin(self.h), "profile_begin")
+
+    def profile_end(self):
+        """Returns {category: (milliseconds, event pairs)} since profile_begin (synchronises the stream)."""
+        n = lib().mixaq_profile_categories()
+        ms, cnt = (C.c_float * n)(), (C.c_int * n)()
+        self.check(lib().mixaq_profile_end(self.h, _stream_ptr(), ms, cnt), "profile_end")
+        return {lib().mixaq_profile_category_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     def close(self):
         if self.h:

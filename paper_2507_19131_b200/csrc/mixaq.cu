@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 namespace mixaq {
 bool ln_dim_supported(int C);
@@ -17,12 +18,22 @@ int g_launches = 0;
 
 using namespace mixaq;
 
+struct ProfRec { int cat; cudaEvent_t e0, e1; };
 struct mixaq_ctx {
   int device;
   int* d_status;
   int launches;
   char err[256];
+  bool profiling;
+  std::vector<ProfRec> prof;          // event pairs recorded since mixaq_profile_begin
+  std::vector<cudaEvent_t> pool;      // events ready for reuse
 };
+
+enum ProfCat { PC_ENERGY = 0, PC_SELECT, PC_LN1, PC_QKV, PC_ATTN, PC_PROJ, PC_LN2, PC_FC1, PC_FC2, PC_COPY,
+               PC_MERGE_GATHER, PC_MERGE_GEMM, PC_COUNT };
+static const char* kProfNames[PC_COUNT] = {"energy", "select", "gather_ln1_quant", "gemm_qkv", "attention",
+                                           "gemm_proj", "ln2_quant", "gemm_fc1_gelu", "gemm_fc2_scatter",
+                                           "copy_pruned", "merge_gather_ln_quant", "gemm_merge"};
 
 namespace {
 
@@ -51,6 +62,24 @@ mixaq_status check_cuda(mixaq_ctx* ctx, const char* where) {
   if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s: %s", where, cudaGetErrorString(e));
   return MIXAQ_CUDA_ERROR;
 }
+
+// Per-kernel CUDA-event timing (only while profiling is on; the events sit on the launching stream).
+struct ProfScope {
+  mixaq_ctx* ctx; cudaStream_t st; cudaEvent_t e1; bool on;
+  ProfScope(mixaq_ctx* c, int cat, cudaStream_t s) : ctx(c), st(s), e1(nullptr), on(c && c->profiling) {
+    if (!on) return;
+    cudaEvent_t ev[2];
+    for (int i = 0; i < 2; ++i) {
+      if (!ctx->pool.empty()) { ev[i] = ctx->pool.back(); ctx->pool.pop_back(); }
+      else if (cudaEventCreate(&ev[i]) != cudaSuccess) { on = false; return; }
+    }
+    cudaEventRecord(ev[0], st);
+    e1 = ev[1];
+    ctx->prof.push_back({cat, ev[0], ev[1]});
+  }
+  ~ProfScope() { if (on) cudaEventRecord(e1, st); }
+};
+#define PROF(cat) ProfScope prof_scope_##cat(ctx, cat, st)
 
 bool bits_ok(int b) { return b == 8 || b == 4 || b == 2; }
 bool aq_ok(const mixaq_aq& q, int bits) {
@@ -165,7 +194,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) {
     cudaGetLastError(); delete c; return MIXAQ_CUDA_ERROR;
   }
@@ -176,6 +205,8 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
 mixaq_status mixaq_destroy(mixaq_ctx* ctx) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   if (ctx->d_status) cudaFree(ctx->d_status);
+  for (auto& r : ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+  for (auto e : ctx->pool) cudaEventDestroy(e);
   delete ctx;
   return MIXAQ_OK;
 }
@@ -189,8 +220,33 @@ mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream) {
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (cudaMemcpyAsync(&h, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess)
-    return check_cuda(ctx, "status read") == MIXAQ_OK ? MIXAQ_CUDA_ERROR : MIXAQ_CUDA_ERROR;
+  { check_cuda(ctx, "status read"); return MIXAQ_CUDA_ERROR; }
   return h == 0 ? MIXAQ_OK : MIXAQ_DEVICE_TIMEOUT;
+}
+
+int mixaq_profile_categories(void) { return PC_COUNT; }
+const char* mixaq_profile_category_name(int cat) { return (cat >= 0 && cat < PC_COUNT) ? kProfNames[cat] : ""; }
+
+mixaq_status mixaq_profile_begin(mixaq_ctx* ctx) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  for (auto& r : ctx->prof) { ctx->pool.push_back(r.e0); ctx->pool.push_back(r.e1); }
+  ctx->prof.clear();
+  ctx->profiling = true;
+  return MIXAQ_OK;
+}
+
+mixaq_status mixaq_profile_end(mixaq_ctx* ctx, void* cuda_stream, float* ms_per_category, int* launches_per_category) {
+  if (!ctx || !ms_per_category || !launches_per_category) return MIXAQ_INVALID_ARG;
+  ctx->profiling = false;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return check_cuda(ctx, "profile_end");
+  for (int i = 0; i < PC_COUNT; ++i) { ms_per_category[i] = 0.f; launches_per_category[i] = 0; }
+  for (auto& r : ctx->prof) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess) { ms_per_category[r.cat] += ms; launches_per_category[r.cat] += 1; }
+    ctx->pool.push_back(r.e0); ctx->pool.push_back(r.e1);
+  }
+  ctx->prof.clear();
+  return check_cuda(ctx, "profile_end");
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -273,14 +329,14 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
 
   // 1. scores and selection
   const int32_t* energy = opts ? opts->energy : nullptr;
-  if (!energy) { launch_energy(x, ws.energy, (long)B * H * W, C, p->score_inv_scale, st); energy = ws.energy; }
+  if (!energy) { PROF(PC_ENERGY); launch_energy(x, ws.energy, (long)B * H * W, C, p->score_inv_scale, st); energy = ws.energy; }
   SelectArgs sa;
   sa.energy = energy; sa.score = ws.score; sa.order = ws.order; sa.cls = ws.cls;
   sa.rowsrc_hi = ws.rowsrc[0]; sa.rowsrc_lo = ws.rowsrc[1]; sa.rowsrc_pr = ws.rowsrc[2];
   sa.win_hi = ws.win[0]; sa.win_lo = ws.win[1];
   sa.B = B; sa.H = H; sa.W = W; sa.shift = p->shift; sa.nwx = g.nwx; sa.nW = g.nW;
   sa.n_hi = g.n_hi; sa.n_lo = g.n_lo; sa.n_pr = g.n_pr; sa.reverse = opts ? opts->reverse : 0;
-  launch_select(sa, st);
+  { PROF(PC_SELECT); launch_select(sa, st); }
   if (sel_out) {
     const size_t n = (size_t)B * g.nW;
     if (sel_out->cls)   cudaMemcpyAsync(sel_out->cls, ws.cls, n, cudaMemcpyDeviceToDevice, st);
@@ -299,7 +355,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     lb[i].src = x; lb[i].rowsrc = ws.rowsrc[i]; lb[i].gamma = brp[i]->ln1_g; lb[i].beta = brp[i]->ln1_b;
     lb[i].out = ws.a[i]; lb[i].q = to_aq(brp[i]->qkv_in); lb[i].M = M[i];
   }
-  launch_ln_quant(lb[0], lb[1], C, st);
+  { PROF(PC_LN1); launch_ln_quant(lb[0], lb[1], C, st); }
 
   // 3. QKV GEMM -> q, k, v codes
   GemmArgs ga;
@@ -310,7 +366,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.qkv[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->qkv_acc : nullptr;
   }
-  launch_gemm(ga, st);
+  { PROF(PC_QKV); launch_gemm(ga, st); }
 
   // 4. window attention
   AttnArgs aa;
@@ -326,7 +382,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ab.so = (1.0f / (float)((1 << brp[i]->bits) - 1)) * brp[i]->v.scale;
     ab.tap_p = tp[i] ? tp[i]->p_codes : nullptr; ab.tap_pv = tp[i] ? tp[i]->pv_acc : nullptr;
   }
-  launch_attention(aa, st);
+  { PROF(PC_ATTN); launch_attention(aa, st); }
 
   // 5. proj GEMM + attention residual -> x1
   ga.w = p->proj.codes; ga.N = C; ga.K = C; ga.mode = EPI_PROJ;
@@ -335,14 +391,14 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = ws.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->proj_acc : nullptr;
   }
-  launch_gemm(ga, st);
+  { PROF(PC_PROJ); launch_gemm(ga, st); }
 
   // 6. LN2 + quantize + pack
   for (int i = 0; i < 2; ++i) {
     lb[i].src = ws.x1[i]; lb[i].rowsrc = nullptr; lb[i].gamma = brp[i]->ln2_g; lb[i].beta = brp[i]->ln2_b;
     lb[i].out = ws.f1[i]; lb[i].q = to_aq(brp[i]->fc1_in); lb[i].M = M[i];
   }
-  launch_ln_quant(lb[0], lb[1], C, st);
+  { PROF(PC_LN2); launch_ln_quant(lb[0], lb[1], C, st); }
 
   // 7. fc1 GEMM + GELU + requantize
   ga.w = p->fc1.codes; ga.N = Hd; ga.K = C; ga.mode = EPI_FC1;
@@ -351,7 +407,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].q0 = to_aq(brp[i]->fc2_in); ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.f2[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc1_acc : nullptr;
   }
-  launch_gemm(ga, st);
+  { PROF(PC_FC1); launch_gemm(ga, st); }
 
   // 8. fc2 GEMM + residual + scatter (reverse shift, crop)
   ga.w = p->fc2.codes; ga.N = C; ga.K = Hd; ga.mode = EPI_FC2;
@@ -360,10 +416,10 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = ws.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc2_acc : nullptr;
   }
-  launch_gemm(ga, st);
+  { PROF(PC_FC2); launch_gemm(ga, st); }
 
   // 9. pruned windows are forwarded unchanged
-  launch_copy_rows(x, y, ws.rowsrc[2], B * g.n_pr * WT, C, st);
+  { PROF(PC_COPY); launch_copy_rows(x, y, ws.rowsrc[2], B * g.n_pr * WT, C, st); }
 
   if (taps) {
     for (int i = 0; i < 2; ++i) {
@@ -404,7 +460,7 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
   MergeGatherArgs mg;
   mg.x = x; mg.gamma = p->ln_g; mg.beta = p->ln_b; mg.out = (uint8_t*)workspace; mg.q = to_aq(p->in);
   mg.B = B; mg.H = H; mg.W = W; mg.C = C;
-  launch_merge_gather(mg, st);
+  { PROF(PC_MERGE_GATHER); launch_merge_gather(mg, st); }
   Carver c(p->prepared);
   float* mult = c.take<float>(N);
   int32_t* zc = c.take<int32_t>(N);
@@ -413,7 +469,7 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
   fill_gemm_branch(ga.br[0], (const uint8_t*)workspace, M, p->in.bits, mult, zc, nullptr);
   ga.br[0].out_f = y;
   fill_gemm_branch(ga.br[1], nullptr, 0, p->in.bits, mult, zc, nullptr);
-  launch_gemm(ga, st);
+  { PROF(PC_MERGE_GEMM); launch_gemm(ga, st); }
   ctx->launches = g_launches;
   return check_cuda(ctx, "merge_forward");
 }
@@ -489,7 +545,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
       cur = mdst; H = (H + 1) / 2; W = (W + 1) / 2;
     }
     const mixaq_block_params* b0 = &p->blocks[blk];
-    launch_energy(cur, ws.energy, (long)B * H * W, b0->dim, b0->score_inv_scale, st);
+    { PROF(PC_ENERGY); launch_energy(cur, ws.energy, (long)B * H * W, b0->dim, b0->score_inv_scale, st); }
     total += 1;
     mixaq_select_opts so; so.energy = ws.energy; so.reverse = 0;
     for (int i = 0; i < d; ++i, ++blk) {
