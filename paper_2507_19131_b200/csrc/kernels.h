@@ -63,9 +63,10 @@ struct GemmArgs {
   const int8_t* w;           // [N][K]
   int N, K, C;               // C: channels per q/k/v section (EPI_QKV)
   int mode;
+  int* status;           // device status word (raised when a bounded wait runs out)
   GemmBranch br[2];
 };
-void launch_gemm(const GemmArgs& g, cudaStream_t st);
+bool launch_gemm(const GemmArgs& g, cudaStream_t st);
 
 // ---- fused window attention ----------------------------------------------------------------------
 struct AttnBranch {

@@ -12,7 +12,6 @@
 namespace mixaq {
 bool ln_dim_supported(int C);
 bool merge_dim_supported(int C);
-void launch_gemm_simple(const GemmArgs& g, cudaStream_t st);
 int g_launches = 0;
 }  // namespace mixaq
 
@@ -359,6 +358,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
 
   // 3. QKV GEMM -> q, k, v codes
   GemmArgs ga;
+  ga.status = ctx->d_status;
   ga.w = p->qkv.codes; ga.N = 3 * C; ga.K = C; ga.C = C; ga.mode = EPI_QKV;
   for (int i = 0; i < 2; ++i) {
     fill_gemm_branch(ga.br[i], ws.a[i], M[i], brp[i]->bits, pr.mult[0][i], pr.zc[0][i], brp[i]->b_qkv);
@@ -366,7 +366,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.qkv[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->qkv_acc : nullptr;
   }
-  { PROF(PC_QKV); launch_gemm(ga, st); }
+  { PROF(PC_QKV); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 4. window attention
   AttnArgs aa;
@@ -391,7 +391,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = ws.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->proj_acc : nullptr;
   }
-  { PROF(PC_PROJ); launch_gemm(ga, st); }
+  { PROF(PC_PROJ); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 6. LN2 + quantize + pack
   for (int i = 0; i < 2; ++i) {
@@ -407,7 +407,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].q0 = to_aq(brp[i]->fc2_in); ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.f2[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc1_acc : nullptr;
   }
-  { PROF(PC_FC1); launch_gemm(ga, st); }
+  { PROF(PC_FC1); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 8. fc2 GEMM + residual + scatter (reverse shift, crop)
   ga.w = p->fc2.codes; ga.N = C; ga.K = Hd; ga.mode = EPI_FC2;
@@ -416,7 +416,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
     ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = ws.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc2_acc : nullptr;
   }
-  { PROF(PC_FC2); launch_gemm(ga, st); }
+  { PROF(PC_FC2); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 9. pruned windows are forwarded unchanged
   { PROF(PC_COPY); launch_copy_rows(x, y, ws.rowsrc[2], B * g.n_pr * WT, C, st); }
@@ -465,11 +465,12 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
   float* mult = c.take<float>(N);
   int32_t* zc = c.take<int32_t>(N);
   GemmArgs ga;
+  ga.status = ctx->d_status;
   ga.w = p->reduction.codes; ga.N = N; ga.K = K; ga.C = N; ga.mode = EPI_MERGE;
   fill_gemm_branch(ga.br[0], (const uint8_t*)workspace, M, p->in.bits, mult, zc, nullptr);
   ga.br[0].out_f = y;
   fill_gemm_branch(ga.br[1], nullptr, 0, p->in.bits, mult, zc, nullptr);
-  { PROF(PC_MERGE_GEMM); launch_gemm(ga, st); }
+  { PROF(PC_MERGE_GEMM); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
   ctx->launches = g_launches;
   return check_cuda(ctx, "merge_forward");
 }
