@@ -146,6 +146,29 @@ size_t       mixaq_merge_workspace_bytes(const mixaq_merge_params* p, int B, int
 mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
                                  int B, int H, int W, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* ---- patch merging without a workspace (the paper has no counterpart: this entry point exists for the way the
+ *      library is deployed, not for the method).  Same result as mixaq_merge_forward, bit for bit, but the
+ *      intermediate code matrix lives in an array built into the library, so the call asks the caller for no
+ *      workspace and allocates nothing itself (no cudaMalloc / cudaFree, no allocating library routine).
+ *      It is meant for callers that cannot obtain device memory where they run the network: a plug-in inside
+ *      an application whose own pool holds the whole device, a frame loop that must not hit the device-wide
+ *      synchronisation an allocation implies, a process whose policy forbids driver allocations after start-up.
+ *      x, y, the parameters and `prepared` are still the caller's, as for mixaq_merge_forward.
+ *      Limits and rules:
+ *        - the code matrix, B*ceil(H/2)*ceil(W/2) rows of 4C*in.bits/8 bytes, must fit in
+ *          MIXAQ_STATIC_SCRATCH_BYTES; larger problems are refused with MIXAQ_WORKSPACE_TOO_SMALL (the text
+ *          of mixaq_last_error names both sizes) before anything is launched;
+ *        - every GPU that loads the library holds MIXAQ_STATIC_SCRATCH_BYTES of device memory until the
+ *          process exits, used or not;
+ *        - the first call on each device looks up the array's device address (with that device current);
+ *          make that first call outside any stream capture;
+ *        - all calls on one device share the one array: two calls whose kernels can overlap on the GPU (different
+ *          streams, no ordering between them) race on it.  Calls ordered on one stream are safe.  The array
+ *          keeps the previous call's bytes; each call rewrites every byte it later reads, so nothing is cleared. ---- */
+#define MIXAQ_STATIC_SCRATCH_BYTES (8u << 20)
+mixaq_status mixaq_merge_forward_static(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
+                                        int B, int H, int W, void* cuda_stream);
+
 /* ---- the backbone: for every stage [merge] -> stage energy -> blocks; one ratio per pair of consecutive
  *      blocks (Section 3.3), optional prune ratio per pair (Section 3.4).  x0 is the [B][H0][W0][C0] map after the
  *      patch-embedding stem; stage_out is a HOST array of num_stages device pointers receiving each stage's final

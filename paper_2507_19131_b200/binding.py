@@ -21,7 +21,7 @@ EXPORTS = [
     "mixaq_merge_prepare", "mixaq_stage_energy", "mixaq_block_workspace_bytes", "mixaq_block_forward",
     "mixaq_merge_workspace_bytes", "mixaq_merge_forward", "mixaq_backbone_workspace_bytes",
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
-    "mixaq_profile_begin", "mixaq_profile_end",
+    "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -311,6 +311,20 @@ def merge_forward(ctx: Context, dm: DeviceMerge, x: torch.Tensor) -> torch.Tenso
     ws = torch.empty(need, dtype=torch.uint8, device=x.device)
     ctx.check(lib().mixaq_merge_forward(ctx.h, C.byref(dm.s), _ptr(x), _ptr(y), B, H, W, _ptr(ws), C.c_size_t(need),
                                         _stream_ptr()), "merge_forward")
+    return y
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def merge_forward_static(ctx: Context, dm: DeviceMerge, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """mixaq_merge_forward_static: patch merging for callers that cannot allocate device memory where they run
+    the network (the intermediate lives in an array built into the library, at most STATIC_SCRATCH_BYTES).
+    The caller passes the output tensor; nothing is allocated here or in the library."""
+    B, H, W, Cc = x.shape
+    assert tuple(y.shape) == (B, (H + 1) // 2, (W + 1) // 2, 2 * Cc) and y.dtype == torch.float32 and y.is_contiguous()
+    ctx.check(lib().mixaq_merge_forward_static(ctx.h, C.byref(dm.s), _ptr(x), _ptr(y), B, H, W, _stream_ptr()),
+              "merge_forward_static")
     return y
 
 

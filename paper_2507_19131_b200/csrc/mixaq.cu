@@ -28,6 +28,15 @@ struct mixaq_ctx {
   std::vector<cudaEvent_t> pool;      // events ready for reuse
 };
 
+namespace mixaq {
+// accessors for translation units that do not see the context's layout
+int* ctx_status_word(mixaq_ctx* ctx) { return ctx->d_status; }
+void ctx_note(mixaq_ctx* ctx, const char* msg, int launches) {
+  if (msg) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
+  ctx->launches = launches;
+}
+}  // namespace mixaq
+
 enum ProfCat { PC_ENERGY = 0, PC_SELECT, PC_LN1, PC_QKV, PC_ATTN, PC_PROJ, PC_LN2, PC_FC1, PC_FC2, PC_COPY,
                PC_MERGE_GATHER, PC_MERGE_GEMM, PC_COUNT };
 static const char* kProfNames[PC_COUNT] = {"energy", "select", "gather_ln1_quant", "gemm_qkv", "attention",
