@@ -3,10 +3,33 @@
 //   S_int = (q - z_q)(k - z_k)^T  (int32)  ->  S = fma(S_int, s_q*s_k/sqrt(d), relpos_bias) [+ shift mask]
 //   P = softmax_row(S) in binary32  ->  P codes (unsigned, step 1/(2^b-1))
 //   O_int = P_codes (v - z_v) (int32)  ->  O = O_int * s_p*s_v  ->  codes of the proj input quantizer.
-// One CTA per (window slot, head); thread i owns query row i.
+//
+// One warp per (window slot, head).  Both products run on the integer tensor cores of the warp
+// (mma.sync m16n8k32, u8 x u8 -> s32; 49 tokens padded to 64 query rows x 56 key columns).  The 49 x 32 problem is
+// far too small for a 128-row tcgen05 tile and is bound by the softmax arithmetic, not by the MMA rate.
+// The softmax runs on the accumulator fragments: a quad of lanes holds one row, lane t of the quad owns columns
+// 8g+2t, 8g+2t+1 -- exactly the four interleaved partial sums of the numeric contract.  The P codes go from
+// accumulator layout to A-operand layout without leaving the thread: the key index of P.V is permuted
+// consistently on both operands (V^T is staged in shared memory with its columns in that order).
 #include "kernels.h"
 
 namespace mixaq {
+
+namespace {
+
+constexpr int ATT_WARPS = 4;
+constexpr int QK_LD = 12;     // words per staged q / k row (8 used; 12 keeps fragment reads conflict-free)
+constexpr int VT_LD = 20;     // words per row of V^T (16 used)
+
+struct WarpSmem {
+  uint32_t q[64][QK_LD];      // query rows (one code per byte), rows >= 49 zero
+  uint32_t k[56][QK_LD];      // key rows
+  uint32_t vt[32][VT_LD];     // V^T: row e, 64 key positions in the permuted order of pos()
+  int rq[64];                 // per query row:  -z_k * sum_d q + 32 z_q z_k
+  int ck[56];                 // per key column: -z_q * sum_d k
+  uint32_t o[16][8];          // staging of 16 output rows x 32 codes (one per byte)
+  uint8_t reg[64];            // shift region of every token
+};
 
 __device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
   int d;
@@ -14,131 +37,276 @@ __device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
   return d;
 }
 
+__device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 __device__ __forceinline__ int shift_region(int pos, int L, int shift) {
   return pos < L - WS ? 0 : (pos < L - shift ? 1 : 2);
 }
 
-__global__ void __launch_bounds__(64) k_attention(AttnArgs a) {
-  __shared__ uint32_t s_q[WT][8], s_k[WT][8], s_v[WT][8];
-  __shared__ int s_reg[WT], s_ksum[WT];
+// Position of key j inside V^T rows: within each group of 32 keys, the MMA's k index 4t+u (u = 0..3) of lane t
+// holds the P code of accumulator tile 2*0+(u>>1), column 2t+(u&1); k index 16+4t+u that of tiles 2, 3.
+__device__ __forceinline__ int pos(int j) {
+  const int jj = j & 31, nt = jj >> 3, c = jj & 7, t = c >> 1, u0 = c & 1;
+  const int kappa = nt < 2 ? 4 * t + 2 * nt + u0 : 16 + 4 * t + 2 * (nt - 2) + u0;
+  return (j & 32) + kappa;
+}
+
+// pack eight bytes (two words) into eight nibbles, little end first
+__device__ __forceinline__ uint32_t pack_nibbles(uint32_t lo, uint32_t hi) {
+  const uint32_t x = __byte_perm(lo, hi, 0x6420);   // codes 0, 2, 4, 6
+  const uint32_t y = __byte_perm(lo, hi, 0x7531);   // codes 1, 3, 5, 7
+  return x | (y << 4);
+}
+// eight nibbles -> eight 2-bit codes in the low half
+__device__ __forceinline__ uint32_t squeeze_pairs(uint32_t t) {
+  t = (t | (t >> 2)) & 0x0F0F0F0Fu;
+  t = (t | (t >> 4)) & 0x00FF00FFu;
+  t = (t | (t >> 8)) & 0x0000FFFFu;
+  return t;
+}
+
+template <bool SHIFTED>
+__global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
+  __shared__ __align__(16) WarpSmem smem_all[ATT_WARPS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
   const int slots_hi = a.br[0].slots;
-  int slot = blockIdx.x / a.heads, h = blockIdx.x - slot * a.heads;
+  const long wg = (long)blockIdx.x * ATT_WARPS + warp;
+  if (wg >= (long)(slots_hi + a.br[1].slots) * a.heads) return;
+  int slot = (int)(wg / a.heads);
+  const int h = (int)(wg - (long)slot * a.heads);
   const bool is_hi = slot < slots_hi;
   const AttnBranch& br = is_hi ? a.br[0] : a.br[1];
   if (!is_hi) slot -= slots_hi;
+  WarpSmem& sm = smem_all[warp];
   const int bits = br.bits, C = a.C;
   const long row_bytes = (long)3 * C * bits / 8;
-  const int tid = threadIdx.x;
-
-  // stage q, k, v of this head (32 codes each per token), unpacked to bytes
-  for (int i = tid; i < 3 * WT; i += blockDim.x) {
-    int sec = i / WT, t = i - sec * WT;
-    const uint8_t* src = br.qkv + ((long)slot * WT + t) * row_bytes + (long)(sec * C + h * HEAD_DIM) * bits / 8;
-    uint32_t w[8];
-    load_codes_32(src, bits, w);
-    uint32_t (*dst)[8] = sec == 0 ? s_q : (sec == 1 ? s_k : s_v);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) dst[t][e] = w[e];
-  }
-  if (tid < WT) {
-    int reg = 0;
-    if (a.shift > 0) {
-      int w = br.win[slot];
-      int wy = w / a.nwx, wx = w - wy * a.nwx;
-      int i = tid / WS, j = tid - i * WS;
-      reg = shift_region(wy * WS + i, a.Hp, a.shift) * 3 + shift_region(wx * WS + j, a.Wp, a.shift);
-    }
-    s_reg[tid] = reg;
-  }
-  __syncthreads();
-  if (tid < WT) {
-    int ks = 0;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) ks = dp4a_uu(s_k[tid][e], 0x01010101u, ks);
-    s_ksum[tid] = ks;
-  }
-  __syncthreads();
-  if (tid >= WT) return;
-
-  const int i = tid;
   const int zq = br.q.zp, zk = br.k.zp, zv = br.v.zp;
-  uint32_t qw[8];
-  int qsum = 0;
+
+  // ---- stage q, k (rows) and v (transposed, permuted) of this head, one code per byte ----
+  int wy = 0, wx = 0;
+  if (SHIFTED) { const int w = br.win[slot]; wy = w / a.nwx; wx = w - wy * a.nwx; }
 #pragma unroll
-  for (int e = 0; e < 8; ++e) { qw[e] = s_q[i][e]; qsum = dp4a_uu(qw[e], 0x01010101u, qsum); }
-  const float* relb = a.relbias + ((long)h * WT + i) * WT;
-  const int my_reg = s_reg[i];
-  float lg[WT];
-  float mx = -3.0e38f;
+  for (int half = 0; half < 2; ++half) {
+    const int r = lane + 32 * half;
+    const int p = pos(r);
+    uint8_t* vtb = reinterpret_cast<uint8_t*>(&sm.vt[0][0]);
+    if (r < WT) {
+      const uint8_t* src = br.qkv + ((long)slot * WT + r) * row_bytes + (long)(h * HEAD_DIM) * bits / 8;
+      uint32_t w[8];
+      load_codes_32(src, bits, w);
+      int s = 0;
 #pragma unroll
-  for (int j = 0; j < WT; ++j) {
-    int dot = 0;
+      for (int e = 0; e < 8; ++e) s = dp4a_uu(w[e], 0x01010101u, s);
+      *reinterpret_cast<uint4*>(&sm.q[r][0]) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(&sm.q[r][4]) = make_uint4(w[4], w[5], w[6], w[7]);
+      sm.rq[r] = -zk * s + HEAD_DIM * zq * zk;
+      load_codes_32(src + (long)C * bits / 8, bits, w);
+      s = 0;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) dot = dp4a_uu(qw[e], s_k[j][e], dot);
-    int s_int = dot - zk * qsum - zq * s_ksum[j] + HEAD_DIM * zq * zk;
-    float v = __fmaf_rn(__int2float_rn(s_int), br.alpha, __ldg(relb + j));
-    if (a.shift > 0) v = __fadd_rn(v, s_reg[j] != my_reg ? -100.0f : 0.0f);
-    lg[j] = v;
-    mx = fmaxf(mx, v);
-  }
-  const float kLog2e = 1.44269504088896340736f;
+      for (int e = 0; e < 8; ++e) s = dp4a_uu(w[e], 0x01010101u, s);
+      *reinterpret_cast<uint4*>(&sm.k[r][0]) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(&sm.k[r][4]) = make_uint4(w[4], w[5], w[6], w[7]);
+      sm.ck[r] = -zq * s;
+      load_codes_32(src + (long)2 * C * bits / 8, bits, w);
 #pragma unroll
-  for (int j = 0; j < WT; ++j) lg[j] = exp2_core(fmaxf(__fmul_rn(__fsub_rn(lg[j], mx), kLog2e), -125.0f));
-  // sum: four interleaved partials (columns 8g+2t, 8g+2t+1 -> partial t), then (p0+p1)+(p2+p3)
-  float part[4];
-#pragma unroll
-  for (int t = 0; t < 4; ++t) {
-    float p = 0.0f;
-#pragma unroll
-    for (int g = 0; g < 7; ++g)
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        int j = 8 * g + 2 * t + u;
-        if (j < WT) p = __fadd_rn(p, lg[j]);
+      for (int e = 0; e < 32; ++e) vtb[e * (VT_LD * 4) + p] = (uint8_t)(w[e >> 2] >> (8 * (e & 3)));
+      int reg = 0;
+      if (SHIFTED) {
+        const int i = r / WS, j = r - i * WS;
+        reg = shift_region(wy * WS + i, a.Hp, a.shift) * 3 + shift_region(wx * WS + j, a.Wp, a.shift);
       }
-    part[t] = p;
-  }
-  float sum = __fadd_rn(__fadd_rn(part[0], part[1]), __fadd_rn(part[2], part[3]));
-  float inv = __fdiv_rn(1.0f, sum);
-  const int pmax = (1 << bits) - 1;
-  AQ pq; pq.scale = 0.f; pq.inv_scale = (float)pmax; pq.zpf = 0.0f; pq.qmaxf = (float)pmax; pq.zp = 0; pq.bits = bits;
-  uint32_t pc[WT];
-  int psum = 0;
+      sm.reg[r] = (uint8_t)reg;
+    } else {
+      *reinterpret_cast<uint4*>(&sm.q[r][0]) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(&sm.q[r][4]) = make_uint4(0, 0, 0, 0);
+      sm.rq[r] = 0;
+      sm.reg[r] = 0;
+      if (r < 56) {
+        *reinterpret_cast<uint4*>(&sm.k[r][0]) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(&sm.k[r][4]) = make_uint4(0, 0, 0, 0);
+        sm.ck[r] = 0;
+      }
 #pragma unroll
-  for (int j = 0; j < WT; ++j) { pc[j] = quant_code(__fmul_rn(lg[j], inv), pq); psum += (int)pc[j]; }
-  if (br.tap_p) {
-    uint8_t* tp = br.tap_p + (((long)slot * a.heads + h) * WT + i) * WT;
-#pragma unroll
-    for (int j = 0; j < WT; ++j) tp[j] = (uint8_t)pc[j];
-  }
-  int o_int[HEAD_DIM];
-#pragma unroll
-  for (int e = 0; e < HEAD_DIM; ++e) o_int[e] = -zv * psum;
-#pragma unroll
-  for (int j = 0; j < WT; ++j) {
-#pragma unroll
-    for (int e8 = 0; e8 < 8; ++e8) {
-      uint32_t vw = s_v[j][e8];
-#pragma unroll
-      for (int b = 0; b < 4; ++b) o_int[e8 * 4 + b] += (int)pc[j] * (int)((vw >> (8 * b)) & 0xFFu);
+      for (int e = 0; e < 32; ++e) vtb[e * (VT_LD * 4) + p] = 0;
     }
   }
-  const long m = (long)slot * WT + i;
-  if (br.tap_pv) {
+  __syncwarp();
+
+  // ---- key fragments, per-column terms and regions of this lane's 14 columns (fixed over the query tiles) ----
+  uint32_t kb0[7], kb1[7];
+  int ckj[7][2];
+  uint32_t regj_lo = 0, regj_hi = 0;          // 4 bits per column: columns of tiles 0..3 in lo, 4..6 in hi
 #pragma unroll
-    for (int e = 0; e < HEAD_DIM; ++e) br.tap_pv[m * C + h * HEAD_DIM + e] = o_int[e];
+  for (int nt = 0; nt < 7; ++nt) {
+    kb0[nt] = sm.k[8 * nt + g][t];
+    kb1[nt] = sm.k[8 * nt + g][4 + t];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int j = 8 * nt + 2 * t + u;
+      ckj[nt][u] = sm.ck[j];
+      if (SHIFTED) {
+        const uint32_t rj = sm.reg[j];
+        if (nt < 4) regj_lo |= rj << (4 * (2 * nt + u)); else regj_hi |= rj << (4 * (2 * (nt - 4) + u));
+      }
+    }
   }
-  uint32_t oc[32];
-  AQ oq = br.o;
+  const float alpha = br.alpha, so = br.so;
+  const int pmax = (1 << bits) - 1;
+  const float pmaxf = (float)pmax;
+  const AQ oq = br.o;
+  const float kLog2e = 1.44269504088896340736f;
+  const float4* relf = reinterpret_cast<const float4*>(a.relbias) + (long)h * (4 * 7 * 32) + lane;
+  const long m_base = (long)slot * WT;
+  const long out_row_bytes = (long)C * bits / 8;
+
+#pragma unroll 1
+  for (int mt = 0; mt < 4; ++mt) {
+    // ---- S = Q K^T for 16 query rows ----
+    uint32_t qa[4];
+    qa[0] = sm.q[16 * mt + g][t];     qa[1] = sm.q[16 * mt + g + 8][t];
+    qa[2] = sm.q[16 * mt + g][4 + t]; qa[3] = sm.q[16 * mt + g + 8][4 + t];
+    int c[7][4];
 #pragma unroll
-  for (int e = 0; e < HEAD_DIM; ++e) oc[e] = quant_code(__fmul_rn(__int2float_rn(o_int[e]), br.so), oq);
-  store_codes_32(br.out + m * ((long)C * bits / 8) + (long)h * HEAD_DIM * bits / 8, oc, bits);
+    for (int nt = 0; nt < 7; ++nt) {
+      c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0;
+      mma_u8(c[nt], qa, kb0[nt], kb1[nt]);
+    }
+    const int nrows = mt < 3 ? 2 : 1;           // rows 56..63 do not exist: skip the upper half of the last tile
+    uint32_t pa[2][4];                          // P codes as A fragments of the two 32-key steps
+    int psum[2] = {0, 0};
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) { pa[ks][0] = pa[ks][1] = pa[ks][2] = pa[ks][3] = 0; }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (r < nrows) {
+        const int i = 16 * mt + g + 8 * r;
+        const int rqi = sm.rq[i];
+        uint32_t xlo = 0, xhi = 0;
+        if (SHIFTED) { const uint32_t ri = sm.reg[i] * 0x11111111u; xlo = regj_lo ^ ri; xhi = regj_hi ^ ri; }
+        float lg[7][2];
+        float mx = -3.0e38f;
+#pragma unroll
+        for (int nt = 0; nt < 7; ++nt) {
+          const float4 rb = __ldg(relf + (mt * 7 + nt) * 32);
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int s_int = c[nt][2 * r + u] + rqi + ckj[nt][u];
+            const float rel = r == 0 ? (u == 0 ? rb.x : rb.y) : (u == 0 ? rb.z : rb.w);
+            float v = __fmaf_rn(__int2float_rn(s_int), alpha, rel);
+            if (SHIFTED) {
+              const uint32_t x = nt < 4 ? (xlo >> (4 * (2 * nt + u))) & 15u : (xhi >> (4 * (2 * (nt - 4) + u))) & 15u;
+              v = __fadd_rn(v, x != 0 ? -100.0f : 0.0f);
+            }
+            lg[nt][u] = v;
+            const bool valid = nt < 6 || (t == 0 && u == 0);       // key columns 49..55 do not exist
+            if (valid) mx = fmaxf(mx, v);
+          }
+        }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        // exponentials and this lane's partial sum in column order (the partial of index t of the contract)
+        float part = 0.0f;
+#pragma unroll
+        for (int nt = 0; nt < 7; ++nt)
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const bool valid = nt < 6 || (t == 0 && u == 0);
+            float e = exp2_core(fmaxf(__fmul_rn(__fsub_rn(lg[nt][u], mx), kLog2e), -125.0f));
+            e = valid ? e : 0.0f;
+            lg[nt][u] = e;
+            part = __fadd_rn(part, e);
+          }
+        const float s1 = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, 1));
+        const float sum = __fadd_rn(s1, __shfl_xor_sync(0xffffffffu, s1, 2));
+        const float inv = __fdiv_rn(1.0f, sum);
+        // P codes: clamp(rne(p * pmax), 0, pmax); byte u of A register (ks, r [+2]) is tile 4ks + [2 +] (u>>1), column u&1
+        int ps = 0;
+#pragma unroll
+        for (int nt = 0; nt < 7; ++nt) {
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            float tq = __fmul_rn(__fmul_rn(lg[nt][u], inv), pmaxf);
+            tq = fminf(fmaxf(tq, 0.0f), pmaxf);
+            const uint32_t code = __float_as_uint(__fadd_rn(tq, 12582912.0f)) - kMagicBits;
+            ps += (int)code;
+            const int ks = nt >> 2, sub = nt & 3;
+            pa[ks][r + 2 * (sub >> 1)] |= code << (8 * (2 * (sub & 1) + u));
+            if (br.tap_p) {
+              const int j = 8 * nt + 2 * t + u;
+              if (i < WT && j < WT) br.tap_p[(((long)slot * a.heads + h) * WT + i) * WT + j] = (uint8_t)code;
+            }
+          }
+        }
+        ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+        ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+        psum[r] = ps;
+      }
+    }
+    // ---- O = P V for the 16 rows: two 32-key steps, four 8-column tiles of the head dimension ----
+    int d[4][4];
+#pragma unroll
+    for (int ne = 0; ne < 4; ++ne) {
+      d[ne][0] = d[ne][1] = d[ne][2] = d[ne][3] = 0;
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks)
+        mma_u8(d[ne], pa[ks], sm.vt[8 * ne + g][8 * ks + t], sm.vt[8 * ne + g][8 * ks + 4 + t]);
+    }
+    __syncwarp();                               // the previous tile's rows have left the staging area
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int i = 16 * mt + g + 8 * r;
+#pragma unroll
+      for (int ne = 0; ne < 4; ++ne) {
+        uint32_t two = 0;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int o_int = d[ne][2 * r + u] - zv * psum[r];
+          if (br.tap_pv && r < nrows && i < WT) br.tap_pv[(m_base + i) * C + h * HEAD_DIM + 8 * ne + 2 * t + u] = o_int;
+          const uint32_t code = quant_code(__fmul_rn(__int2float_rn(o_int), so), oq);
+          two |= code << (8 * u);
+        }
+        reinterpret_cast<uint16_t*>(&sm.o[g + 8 * r][0])[4 * ne + t] = (uint16_t)two;
+      }
+    }
+    __syncwarp();
+    if (lane < 16) {
+      const int i = 16 * mt + lane;
+      if (i < WT) {
+        const uint4 w0 = *reinterpret_cast<const uint4*>(&sm.o[lane][0]);
+        const uint4 w1 = *reinterpret_cast<const uint4*>(&sm.o[lane][4]);
+        uint8_t* dst = br.out + (m_base + i) * out_row_bytes + (long)h * HEAD_DIM * bits / 8;
+        if (bits == 8) {
+          reinterpret_cast<uint4*>(dst)[0] = w0;
+          reinterpret_cast<uint4*>(dst)[1] = w1;
+        } else {
+          const uint32_t n0 = pack_nibbles(w0.x, w0.y), n1 = pack_nibbles(w0.z, w0.w);
+          const uint32_t n2 = pack_nibbles(w1.x, w1.y), n3 = pack_nibbles(w1.z, w1.w);
+          if (bits == 4) {
+            reinterpret_cast<uint4*>(dst)[0] = make_uint4(n0, n1, n2, n3);
+          } else {
+            reinterpret_cast<uint2*>(dst)[0] = make_uint2(squeeze_pairs(n0) | (squeeze_pairs(n1) << 16),
+                                                          squeeze_pairs(n2) | (squeeze_pairs(n3) << 16));
+          }
+        }
+      }
+    }
+  }
 }
 
+}  // namespace
+
 void launch_attention(const AttnArgs& a, cudaStream_t st) {
-  int slots = a.br[0].slots + a.br[1].slots;
-  if (slots == 0) return;
-  k_attention<<<slots * a.heads, 64, 0, st>>>(a);
+  const long problems = (long)(a.br[0].slots + a.br[1].slots) * a.heads;
+  if (problems == 0) return;
+  const unsigned grid = (unsigned)((problems + ATT_WARPS - 1) / ATT_WARPS);
+  if (a.shift > 0) k_attention<true><<<grid, ATT_WARPS * 32, 0, st>>>(a);
+  else             k_attention<false><<<grid, ATT_WARPS * 32, 0, st>>>(a);
   ++g_launches;
 }
 

@@ -49,13 +49,46 @@ __device__ __forceinline__ float gelu_f(float v) {
   return __fsub_rn(fmaxf(v, 0.0f), h);
 }
 
-// q = clamp(rne(x*inv_scale) + zp, 0, qmax)
-__device__ __forceinline__ uint32_t quant_code(float x, const AQ& q) {
+// q = clamp(rne(x*inv_scale) + zp, 0, qmax), evaluated without a rounding or conversion instruction:
+// rne is monotone and fixes integers, so clamping BEFORE rounding to the integer bounds [-zp, qmax-zp] gives the
+// same code; adding 1.5*2^23 then rounds to nearest-even exactly (|t| <= 255) and leaves 0x4B400000 + rne(t) in
+// the bit pattern.  quant_magic returns that pattern; the code is pattern - 0x4B400000 + zp.
+constexpr uint32_t kMagicBits = 0x4B400000u;
+__device__ __forceinline__ uint32_t quant_magic(float x, const AQ& q) {
   float t = __fmul_rn(x, q.inv_scale);
-  float r = rintf(t);
-  float c = __fadd_rn(r, q.zpf);
-  c = fminf(fmaxf(c, 0.0f), q.qmaxf);
-  return (uint32_t)__float2int_rz(c);
+  t = fminf(fmaxf(t, -q.zpf), q.qmaxf - q.zpf);
+  return __float_as_uint(__fadd_rn(t, 12582912.0f));
+}
+__device__ __forceinline__ uint32_t quant_code(float x, const AQ& q) {
+  return quant_magic(x, q) - kMagicBits + (uint32_t)q.zp;
+}
+// Additive constant that turns sum_i pattern_i << (bits*i) into the packed word of the codes (the per-code
+// offsets zp - 0x4B400000 are folded into one 32-bit constant; every code fits its field, so nothing carries).
+__device__ __forceinline__ uint32_t pack_const(int zp, int bits) {
+  uint32_t k = (uint32_t)zp - kMagicBits, r = 0;
+  for (int sh = 0; sh < 32; sh += bits) r += k << sh;
+  return r;
+}
+// 32 consecutive codes of one row, given as magic patterns, packed and stored (dst is 32*bits/8-byte aligned).
+template <int BITS>
+__device__ __forceinline__ void store_magic_32(uint8_t* dst, const uint32_t (&m)[32], uint32_t kpack) {
+  constexpr int PER = 32 / BITS, WORDS = BITS;   // codes per word, words per 32 codes
+  uint32_t w[WORDS];
+#pragma unroll
+  for (int i = 0; i < WORDS; ++i) {
+    uint32_t v = kpack;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) v += m[PER * i + e] << (BITS * e);
+    w[i] = v;
+  }
+  if (BITS == 8) {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4 % WORDS], w[5 % WORDS], w[6 % WORDS], w[7 % WORDS]);
+  } else if (BITS == 4) {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+  } else {
+    reinterpret_cast<uint2*>(dst)[0] = make_uint2(w[0], w[1]);
+  }
 }
 
 // Sum over a warp by the butterfly of the contract (offsets 16, 8, 4, 2, 1); every lane ends with the
@@ -137,32 +170,39 @@ __device__ __forceinline__ void store_codes_32(uint8_t* dst, const uint32_t (&c)
   }
 }
 
-// Unpack 32 consecutive codes (one k-group) from packed storage into 32 bytes (eight 32-bit words).
+// Eight 4-bit codes of one word -> eight bytes (two words), little end first: mask the even and the odd nibbles
+// into byte lanes, then interleave them with two byte permutes.
+__device__ __forceinline__ void expand_nibbles(uint32_t v, uint32_t& lo, uint32_t& hi) {
+  const uint32_t x = v & 0x0F0F0F0Fu;            // codes 0, 2, 4, 6
+  const uint32_t y = (v >> 4) & 0x0F0F0F0Fu;     // codes 1, 3, 5, 7
+  lo = __byte_perm(x, y, 0x5140);                // x0 y0 x1 y1
+  hi = __byte_perm(x, y, 0x7362);                // x2 y2 x3 y3
+}
+// Eight 2-bit codes in the low half of v -> eight nibbles (bit spread in three shift-or-mask steps).
+__device__ __forceinline__ uint32_t spread_pairs(uint32_t t) {
+  t = (t | (t << 8)) & 0x00FF00FFu;
+  t = (t | (t << 4)) & 0x0F0F0F0Fu;
+  t = (t | (t << 2)) & 0x33333333u;
+  return t;
+}
+
+// Unpack 32 consecutive codes (one k-group) from packed storage (global or shared) into 32 bytes (eight words).
 __device__ __forceinline__ void load_codes_32(const uint8_t* src, int bits, uint32_t (&w)[8]) {
   if (bits == 8) {
     uint4 a = reinterpret_cast<const uint4*>(src)[0], b = reinterpret_cast<const uint4*>(src)[1];
     w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
   } else if (bits == 4) {
     uint4 a = reinterpret_cast<const uint4*>(src)[0];
-    uint32_t p[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {   // 8 nibbles -> 8 bytes
-      uint32_t v = p[i];
-      uint32_t lo = (v & 0xFu) | ((v & 0xF0u) << 4) | ((v & 0xF00u) << 8) | ((v & 0xF000u) << 12);
-      v >>= 16;
-      uint32_t hi = (v & 0xFu) | ((v & 0xF0u) << 4) | ((v & 0xF00u) << 8) | ((v & 0xF000u) << 12);
-      w[2 * i] = lo; w[2 * i + 1] = hi;
-    }
+    expand_nibbles(a.x, w[0], w[1]);
+    expand_nibbles(a.y, w[2], w[3]);
+    expand_nibbles(a.z, w[4], w[5]);
+    expand_nibbles(a.w, w[6], w[7]);
   } else {
     uint2 a = reinterpret_cast<const uint2*>(src)[0];
-    uint32_t p[2] = {a.x, a.y};
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {   // one byte of 4 codes -> 4 bytes
-        uint32_t v = (p[i] >> (8 * j)) & 0xFFu;
-        w[4 * i + j] = (v & 0x3u) | ((v & 0xCu) << 6) | ((v & 0x30u) << 12) | ((v & 0xC0u) << 18);
-      }
+    expand_nibbles(spread_pairs(a.x & 0xFFFFu), w[0], w[1]);
+    expand_nibbles(spread_pairs(a.x >> 16), w[2], w[3]);
+    expand_nibbles(spread_pairs(a.y & 0xFFFFu), w[4], w[5]);
+    expand_nibbles(spread_pairs(a.y >> 16), w[6], w[7]);
   }
 }
 

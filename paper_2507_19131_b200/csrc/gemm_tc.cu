@@ -3,13 +3,18 @@
 //
 //   D[128 x BN] (TMEM) = A[128 x K] (u8, K-major, shared memory) * W[BN x K]^T (s8, K-major, shared memory)
 //
-// Operand staging: 128-byte-swizzled K-major tiles of 128 codes per row and stage.
-//   - weights and 8-bit activations arrive by TMA (cp.async.bulk.tensor, no multicast), completion on an mbarrier;
-//   - 4-bit / 2-bit activations are read bit-packed from global memory by the producer warps, unpacked to
-//     one code per byte in registers and written straight into the swizzled layout the MMA descriptor expects.
-// One CTA computes one 128 x BN output tile; several CTAs share an SM so that the epilogue of one overlaps the
-// loads and MMAs of another.  Every wait on an mbarrier is bounded; on expiry the CTA raises the status word,
-// drains, frees its tensor memory and returns.
+// Persistent, warp-specialised: one CTA per SM walks over the output tiles t = blockIdx.x, + gridDim.x, ...
+//   warp 0      TMA producer: weight tile and (8-bit branches) activation tile of every k-block into a ring of
+//               128-byte-swizzled K-major stages (cp.async.bulk.tensor, no multicast), completion on mbarriers;
+//   warp 1      MMA issuer: one thread feeds the tensor core; the accumulator alternates between two TMEM
+//               buffers so that the epilogue of tile i overlaps the loads and MMAs of tile i+1;
+//   warps 2-3   unpack producers for 4-bit / 2-bit branches: the bit-packed rows of the k-block arrive by TMA in a
+//               staging slot of the stage; these warps expand them to one code per byte, shared to shared, into
+//               the swizzled layout (rows whose byte pitch is no multiple of 16 cannot be described to the TMA
+//               unit and are read with plain loads instead);
+//   warps 4-11  epilogue: tcgen05.ld (one row per thread, 32 columns per load) + the fused epilogue of the mode.
+// Every wait on an mbarrier is bounded; on expiry the CTA raises the status word, drains, frees its tensor
+// memory and returns.
 #include <cuda.h>
 #include "gemm_epilogue.cuh"
 
@@ -21,16 +26,39 @@ constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int BK = 128;            // codes (bytes) per row and stage = one 128-byte swizzle row
 constexpr int UMMA_K = 32;         // codes per tcgen05.mma kind::i8
 constexpr int A_STAGE_BYTES = BM * BK;
-constexpr int NUM_THREADS = 256;
-constexpr int NUM_PRODUCER_WARPS = 6;          // warps 2..7 unpack sub-byte activations
+constexpr int NUM_THREADS = 384;
+constexpr int NUM_UNPACK_WARPS = 2;            // warps 2..3
+constexpr int NUM_UNPACK_THREADS = NUM_UNPACK_WARPS * 32;
+constexpr int NUM_EPI_WARPS = 8;               // warps 4..11
+constexpr int MAX_BN = 256;
+constexpr int EPI_WARP_COLS = MAX_BN / 2;      // columns one epilogue warp handles per tile (every other 32-group)
+constexpr int MAX_RING = 6;
 constexpr uint32_t MAX_POLLS = 1u << 22;
+constexpr int UNPACK_ITEMS = BM * (BK / UMMA_K) / NUM_UNPACK_THREADS;   // (row, 32-code group) items per thread and stage
 
 struct TcParams {
   GemmArgs g;
   int tiles_m0;          // 128-row tiles of the first (high) branch
-  int n_tiles, BN, k_stages, ring, tmem_cols;
+  int total_tiles, n_tiles, BN, k_blocks, ring, tmem_cols;
+  int packed_bytes;      // bytes of the packed staging slot of a stage (0: no branch stages packed rows by TMA)
+  int tma_packed[2];     // branch i stages its bit-packed rows by TMA (tmA_i then describes the packed matrix)
   int* status;
 };
+
+// shared-memory carve-up (offsets from the 1024-byte aligned base)
+struct SmemLayout {
+  int stage_bytes, ring_bytes, consts_off, stage_off, bars_off, total;
+};
+__host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_bytes) {
+  SmemLayout L;
+  L.stage_bytes = A_STAGE_BYTES + BN * BK + packed_bytes;
+  L.ring_bytes = ring * L.stage_bytes;
+  L.consts_off = L.ring_bytes;                                  // per epilogue warp (zc, mult, bias) x 128 columns
+  L.stage_off = L.consts_off + NUM_EPI_WARPS * 3 * EPI_WARP_COLS * 4;   // per epilogue warp 32 x 36 floats
+  L.bars_off = L.stage_off + NUM_EPI_WARPS * EPI_STAGE_FLOATS * 4;
+  L.total = L.bars_off + (3 * MAX_RING + 4) * 8 + 16;
+  return L;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -56,7 +84,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < MAX_POLLS; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
+    if ((it & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
@@ -102,38 +130,48 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+struct TileCoord { int mt, nt; bool is_hi; };
+__device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int t) {
+  TileCoord c;
+  c.nt = t % p.n_tiles;
+  c.mt = t / p.n_tiles;
+  c.is_hi = c.mt < p.tiles_m0;
+  if (!c.is_hi) c.mt -= p.tiles_m0;
+  return c;
+}
+
 template <int MODE>
-__global__ void __launch_bounds__(NUM_THREADS)
+__global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
           const __grid_constant__ CUtensorMap tmB, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
   uint8_t* smem = smem_raw + (base - raw);
-  const int b_stage_bytes = p.BN * BK;
-  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.ring * stage_bytes);
-  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * p.ring, bar_acc = bar_empty + 8u * p.ring;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.ring + 1);
+  const SmemLayout L = smem_layout(p.BN, p.ring, p.packed_bytes);
+  const int stage_bytes = L.stage_bytes;
+  int32_t* s_consts = reinterpret_cast<int32_t*>(smem + L.consts_off);
+  float* s_stage = reinterpret_cast<float*>(smem + L.stage_off);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars_off);
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * MAX_RING, bar_raw = bar_empty + 8u * MAX_RING;
+  const uint32_t bar_tfull = bar_raw + 8u * MAX_RING, bar_tempty = bar_tfull + 16u;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 3 * MAX_RING + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int nt = blockIdx.x % p.n_tiles;
-  int mt = blockIdx.x / p.n_tiles;
-  const bool is_hi = mt < p.tiles_m0;
-  if (!is_hi) mt -= p.tiles_m0;
-  const GemmBranch& br = is_hi ? p.g.br[0] : p.g.br[1];
-  const CUtensorMap* tmA = is_hi ? &tmA0 : &tmA1;
-  const bool packed = br.a_bits != 8;
   const int K = p.g.K;
-  const int m0 = mt * BM, n0 = nt * p.BN;
+  const int acc_stride = p.tmem_cols >> 1;                     // TMEM columns between the two accumulators
 
   if (tid == 0) {
     for (int s = 0; s < p.ring; ++s) {
-      mbar_init(bar_full + 8u * s, packed ? 1u + NUM_PRODUCER_WARPS : 1u);
-      mbar_init(bar_empty + 8u * s, 1u);
+      mbar_init(bar_full + 8u * s, 1u + NUM_UNPACK_WARPS);      // TMA thread + one arrival per unpack warp
+      mbar_init(bar_empty + 8u * s, 1u);                        // tcgen05.commit
+      mbar_init(bar_raw + 8u * s, 1u);                          // TMA thread: "the unpack warps may touch stage s"
     }
-    mbar_init(bar_acc, 1u);
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, 1u);                        // tcgen05.commit of the tile's last MMA
+      mbar_init(bar_tempty + 8u * a, NUM_EPI_WARPS);            // one arrival per epilogue warp
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -148,81 +186,151 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   const uint32_t tmem_base = *tmem_holder;
 
   if (warp == 0) {
-    // ---- TMA producer: weights always, activations when they are stored one code per byte ----
+    // ---- TMA producer ----
     if (lane == 0) {
-      const uint32_t tx = (uint32_t)b_stage_bytes + (packed ? 0u : (uint32_t)A_STAGE_BYTES);
-      for (int ks = 0; ks < p.k_stages; ++ks) {
-        const int s = ks % p.ring;
-        if (ks >= p.ring && !mbar_wait(bar_empty + 8u * s, ((ks / p.ring) - 1) & 1, abort_flag)) break;
-        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + A_STAGE_BYTES;
-        mbar_arrive_expect_tx(bar_full + 8u * s, tx);
-        tma_load_2d(sb, &tmB, ks * BK, n0, bar_full + 8u * s);
-        if (!packed) tma_load_2d(sa, tmA, ks * BK, m0, bar_full + 8u * s);
+      int it = 0;                                               // running k-block counter over all tiles of this CTA
+      bool ok = true;
+      for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
+        const TileCoord tc = decode_tile(p, t);
+        const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
+        const bool packed = br.a_bits != 8;
+        const bool stage_packed = packed && p.tma_packed[tc.is_hi ? 0 : 1];
+        const CUtensorMap* tmA = tc.is_hi ? &tmA0 : &tmA1;
+        const uint32_t tx = (uint32_t)(p.BN * BK) + (packed ? 0u : (uint32_t)A_STAGE_BYTES);
+        const int pk_row = BK * br.a_bits / 8;                  // packed bytes per row and k-block
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % p.ring;
+          if (it >= p.ring && !mbar_wait(bar_empty + 8u * s, ((it / p.ring) - 1) & 1, abort_flag)) { ok = false; break; }
+          const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + A_STAGE_BYTES, sp = sb + (uint32_t)(p.BN * BK);
+          mbar_arrive_expect_tx(bar_full + 8u * s, tx);
+          tma_load_2d(sb, &tmB, kb * BK, tc.nt * p.BN, bar_full + 8u * s);
+          if (!packed) tma_load_2d(sa, tmA, kb * BK, tc.mt * BM, bar_full + 8u * s);
+          if (stage_packed) {
+            mbar_arrive_expect_tx(bar_raw + 8u * s, (uint32_t)(pk_row * BM));
+            tma_load_2d(sp, tmA, kb * pk_row, tc.mt * BM, bar_raw + 8u * s);
+          } else {
+            mbar_arrive(bar_raw + 8u * s);
+          }
+        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---- MMA issuer: one thread feeds the tensor core ----
+    // ---- MMA issuer ----
     if (lane == 0) {
       const uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int it = 0, lt = 0;
       bool ok = true;
-      for (int ks = 0; ks < p.k_stages && ok; ++ks) {
-        const int s = ks % p.ring;
-        ok = mbar_wait(bar_full + 8u * s, (ks / p.ring) & 1, abort_flag);
-        if (!ok) break;
+      for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, ++lt) {
+        const int a = lt & 1;
+        // wait until the epilogue has drained this accumulator (its use two tiles ago)
+        if (lt >= 2 && !mbar_wait(bar_tempty + 8u * a, ((lt >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + A_STAGE_BYTES;
-        const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
-        const int ksteps = min(BK, K - ks * BK) / UMMA_K;
-        for (int kk = 0; kk < ksteps; ++kk)
-          mma_i8(tmem_base, adesc + (uint64_t)(kk * (UMMA_K >> 4)), bdesc + (uint64_t)(kk * (UMMA_K >> 4)), idesc,
-                 (ks > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(bar_empty + 8u * s);          // frees the ring slot when these MMAs have read it
-      }
-      if (ok) mma_commit(bar_acc);               // accumulator complete
-    }
-    __syncwarp();
-  } else if (packed) {
-    // ---- unpack producers: bit-packed rows -> one code per byte, written in the swizzled layout ----
-    const int ptid = tid - 64;                   // 0..191
-    const int abits = br.a_bits;
-    const long row_bytes = (long)K * abits / 8;
-    for (int ks = 0; ks < p.k_stages; ++ks) {
-      const int s = ks % p.ring;
-      if (ks >= p.ring && !mbar_wait(bar_empty + 8u * s, ((ks / p.ring) - 1) & 1, abort_flag)) break;
-      uint8_t* sa = smem + (size_t)s * stage_bytes;
-      const int kgroups = min(BK, K - ks * BK) / UMMA_K;       // 32-code groups in this stage
-      for (int item = ptid; item < BM * kgroups; item += NUM_PRODUCER_WARPS * 32) {
-        const int r = item / kgroups, kg = item - r * kgroups;
-        const long m = (long)m0 + r;
-        if (m < br.M) {
-          uint32_t w[8];
-          load_codes_32(br.a + m * row_bytes + (long)(ks * BK + kg * UMMA_K) * abits / 8, abits, w);
-          uint8_t* rowp = sa + (r >> 3) * 1024 + (r & 7) * 128;
-          const int c0 = (2 * kg) ^ (r & 7), c1 = (2 * kg + 1) ^ (r & 7);
-          *reinterpret_cast<uint4*>(rowp + c0 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(rowp + c1 * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_stride);
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % p.ring;
+          if (!mbar_wait(bar_full + 8u * s, (it / p.ring) & 1, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + A_STAGE_BYTES;
+          const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+          const int ksteps = min(BK, K - kb * BK) / UMMA_K;
+          for (int kk = 0; kk < ksteps; ++kk)
+            mma_i8(d_tmem, adesc + (uint64_t)(kk * (UMMA_K >> 4)), bdesc + (uint64_t)(kk * (UMMA_K >> 4)), idesc,
+                   (kb > 0 || kk > 0) ? 1u : 0u);
+          mma_commit(bar_empty + 8u * s);          // frees the ring slot when these MMAs have read it
         }
+        if (ok) mma_commit(bar_tfull + 8u * a);    // accumulator complete
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA proxy
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_full + 8u * s);
     }
     __syncwarp();
+  } else if (warp < 4) {
+    // ---- unpack producers: bit-packed rows -> one code per byte, written in the swizzled layout ----
+    const int ptid = tid - 64;                   // 0..63
+    int it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
+      const TileCoord tc = decode_tile(p, t);
+      const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
+      const int abits = br.a_bits;
+      const bool packed = abits != 8;
+      const bool staged = packed && p.tma_packed[tc.is_hi ? 0 : 1];
+      const long row_bytes = (long)K * abits / 8;
+      const long m0 = (long)tc.mt * BM;
+      const int grp_bytes = UMMA_K * abits / 8;                 // packed bytes of one 32-code group
+      for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+        const int s = it % p.ring;
+        // the TMA thread arrives on raw[s] once it owns the stage (and, when staged, the packed bytes have landed)
+        if (!mbar_wait(bar_raw + 8u * s, (it / p.ring) & 1, abort_flag)) { ok = false; break; }
+        if (packed) {
+          uint8_t* sa = smem + (size_t)s * stage_bytes;
+          const uint8_t* sp = sa + A_STAGE_BYTES + p.BN * BK;
+          const int kgroups = min(BK, K - kb * BK) / UMMA_K;
+          // item i of this thread: row r = (ptid + 64*i) / 4, 32-code group kg = (ptid + 64*i) % 4
+#pragma unroll
+          for (int i = 0; i < UNPACK_ITEMS; ++i) {
+            const int item = ptid + NUM_UNPACK_THREADS * i;
+            const int r = item >> 2, kg = item & 3;
+            uint32_t w[8];
+            bool have = true;
+            if (staged) {
+              // rows and columns outside the matrix were zero-filled by the TMA unit
+              load_codes_32(sp + item * grp_bytes, abits, w);
+            } else {
+              have = kg < kgroups && m0 + r < br.M;
+              if (have) load_codes_32(br.a + (m0 + r) * row_bytes + (long)(kb * BK + kg * UMMA_K) * abits / 8, abits, w);
+            }
+            if (have) {
+              uint8_t* rowp = sa + (r >> 3) * 1024 + (r & 7) * 128;
+              const int c0 = (2 * kg) ^ (r & 7), c1 = (2 * kg + 1) ^ (r & 7);
+              *reinterpret_cast<uint4*>(rowp + c0 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(rowp + c1 * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA proxy
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_full + 8u * s);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).., column groups e/4, e/4+2, ... ----
+    const int e = warp - 4, q = warp & 3, half = e >> 2;
+    float* stage = s_stage + e * EPI_STAGE_FLOATS;
+    int32_t* c_zc = s_consts + e * 3 * EPI_WARP_COLS;
+    float* c_mult = reinterpret_cast<float*>(c_zc + EPI_WARP_COLS);
+    float* c_bias = c_mult + EPI_WARP_COLS;
+    int lt = 0;
+    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++lt) {
+      const TileCoord tc = decode_tile(p, t);
+      const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
+      const int a = lt & 1;
+      const int n0 = tc.nt * p.BN;
+      // per-column constants of this warp's column groups, in the warp's own shared-memory slot
+      // (no CTA-wide barrier: the only waits of this kernel are the bounded mbarrier waits)
+      __syncwarp();
+      for (int grp = half, j = 0; grp < p.BN / 32; grp += 2, ++j) {
+        const int n = n0 + grp * 32 + lane;
+        c_zc[j * 32 + lane] = __ldg(br.zc + n);
+        c_mult[j * 32 + lane] = __ldg(br.mult + n);
+        if (MODE != EPI_MERGE) c_bias[j * 32 + lane] = __ldg(br.bias + n);
+      }
+      __syncwarp();
+      if (!mbar_wait(bar_tfull + 8u * a, (lt >> 1) & 1, abort_flag)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      ColConsts cc; cc.zc = c_zc; cc.mult = c_mult; cc.bias = c_bias;
+      const long row0 = (long)tc.mt * BM + q * 32;
+      for (int grp = half, j = 0; grp < p.BN / 32; grp += 2, ++j) {
+        int32_t acc[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_stride + grp * 32), acc);
+        epilogue_row32<MODE>(br, p.g.N, p.g.C, row0, lane, n0 + grp * 32, j * 32, cc, acc, stage);
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8u * a);
+    }
   }
 
-  // ---- epilogue: all 8 warps; warp w reads TMEM lanes 32*(w%4).., column groups w/4, w/4+2, ... ----
-  const bool acc_ok = mbar_wait(bar_acc, 0, abort_flag);
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  if (acc_ok) {
-    const int q = warp & 3;
-    const long m = (long)m0 + q * 32 + lane;
-    for (int grp = warp >> 2; grp < p.BN / 32; grp += 2) {
-      int32_t acc[32];
-      tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(grp * 32), acc);
-      if (m < br.M) epilogue_row32<MODE>(br, p.g.N, p.g.C, m, n0 + grp * 32, acc);
-    }
-  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (*abort_flag) {
@@ -257,24 +365,43 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D byte matrix [rows][K] (K contiguous), box = box_rows x 128 bytes, 128-byte swizzle, zero fill outside
-bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
+// 2-D byte matrix [rows][row_bytes] (bytes of a row contiguous), box = box_rows x box_bytes, zero fill outside.
+// swizzled: 128-byte swizzle for MMA operand tiles (box_bytes = 128); otherwise a plain row-major box.
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t row_bytes, uint32_t box_rows,
+              uint32_t box_bytes = BK, bool swizzled = true) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  cuuint64_t dims[2] = {K, rows};
-  cuuint64_t strides[1] = {K};
-  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  cuuint64_t dims[2] = {row_bytes, rows};
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {box_bytes, box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzled ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int pick_bn(int N) {
-  // the widest tile <= 256 that divides N and is a multiple of 32 (epilogue groups) -- and of 16 (MMA N)
-  for (int bn = 256; bn >= 32; bn -= 32)
-    if (N % bn == 0) return bn;
-  return 0;
+int num_sms() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+// Tile width: a multiple of 32 (epilogue groups) that divides N, at most 256; among those, the one that needs the
+// fewest "waves x (columns per tile + fixed per-tile work)" on this many SMs.
+int pick_bn(int N, int m_tiles, int sms) {
+  int best = 0; long best_cost = 0;
+  for (int bn = 32; bn <= MAX_BN; bn += 32) {
+    if (N % bn) continue;
+    const long tiles = (long)m_tiles * (N / bn);
+    const long waves = (tiles + sms - 1) / sms;
+    const long cost = waves * (bn + 48);
+    if (!best || cost <= best_cost) { best = bn; best_cost = cost; }
+  }
+  return best;
 }
 
 template <int MODE>
@@ -283,51 +410,62 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   p.g = g; p.status = status;
   const int t0 = (g.br[0].M + BM - 1) / BM, t1 = (g.br[1].M + BM - 1) / BM;
   if (t0 + t1 == 0) return true;
+  if (g.N % 32 || g.K % UMMA_K) return false;
+  const int sms = num_sms();
   p.tiles_m0 = t0;
-  p.BN = pick_bn(g.N);
-  if (p.BN == 0 || g.K % UMMA_K) return false;
+  p.BN = pick_bn(g.N, t0 + t1, sms);
+  if (p.BN == 0) return false;
   p.n_tiles = g.N / p.BN;
-  p.k_stages = (g.K + BK - 1) / BK;
-  p.ring = p.k_stages < 4 ? p.k_stages : 4;
-  const int stage_bytes = A_STAGE_BYTES + p.BN * BK;
-  while (p.ring > 1 && p.ring * stage_bytes > 200 * 1024) --p.ring;
-  p.tmem_cols = p.BN <= 32 ? 32 : (p.BN <= 64 ? 64 : (p.BN <= 128 ? 128 : 256));
+  p.total_tiles = (t0 + t1) * p.n_tiles;
+  p.k_blocks = (g.K + BK - 1) / BK;
+  // packed branches whose row pitch the TMA unit accepts (a multiple of 16 bytes) are staged by TMA
+  p.packed_bytes = 0;
+  for (int i = 0; i < 2; ++i) {
+    const int bits = g.br[i].a_bits;
+    p.tma_packed[i] = g.br[i].M > 0 && bits != 8 && ((long)g.K * bits / 8) % 16 == 0;
+    if (p.tma_packed[i]) p.packed_bytes = BM * (BK / 2);        // room for the widest packed format (4 bit)
+  }
+  p.ring = MAX_RING;
+  while (p.ring > 2 && smem_layout(p.BN, p.ring, p.packed_bytes).total + 1024 > 220 * 1024) --p.ring;
+  p.tmem_cols = 32;
+  while (p.tmem_cols < 2 * p.BN) p.tmem_cols <<= 1;
   CUtensorMap mA[2], mB;
   memset(mA, 0, sizeof(mA));
   for (int i = 0; i < 2; ++i) {
-    // branches with packed activations, or without rows, get a valid dummy map of the weights (never used)
-    const bool use = g.br[i].M > 0 && g.br[i].a_bits == 8;
-    if (!make_map(&mA[i], use ? (const void*)g.br[i].a : (const void*)g.w, use ? (uint64_t)g.br[i].M : (uint64_t)g.N,
-                  (uint64_t)g.K, use ? BM : (uint32_t)p.BN))
-      return false;
+    const GemmBranch& b = g.br[i];
+    bool ok;
+    if (b.M > 0 && b.a_bits == 8)
+      ok = make_map(&mA[i], b.a, (uint64_t)b.M, (uint64_t)g.K, BM);
+    else if (p.tma_packed[i])
+      ok = make_map(&mA[i], b.a, (uint64_t)b.M, (uint64_t)g.K * b.a_bits / 8, BM, (uint32_t)(BK * b.a_bits / 8), false);
+    else   // no rows, or rows read with plain loads: a valid map of the weights that is never used
+      ok = make_map(&mA[i], g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN);
+    if (!ok) return false;
   }
   if (!make_map(&mB, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN)) return false;
-  const size_t smem = (size_t)p.ring * stage_bytes + 1024 /*alignment slack*/ + (2 * p.ring + 1) * 8 + 16;
+  const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes).total + 1024 /*alignment slack*/;
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(k_gemm_tc<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     attr_set = true;
   }
-  k_gemm_tc<MODE><<<(t0 + t1) * p.n_tiles, NUM_THREADS, smem, st>>>(mA[0], mA[1], mB, p);
+  const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  k_gemm_tc<MODE><<<grid, NUM_THREADS, smem, st>>>(mA[0], mA[1], mB, p);
   ++g_launches;
   return true;
 }
 
 }  // namespace
 
-bool launch_gemm_tc(const GemmArgs& g, int* status, cudaStream_t st) {
+bool launch_gemm(const GemmArgs& g, cudaStream_t st) {
   switch (g.mode) {
-    case EPI_QKV:   return launch_mode<EPI_QKV>(g, status, st);
-    case EPI_PROJ:  return launch_mode<EPI_PROJ>(g, status, st);
-    case EPI_FC1:   return launch_mode<EPI_FC1>(g, status, st);
-    case EPI_FC2:   return launch_mode<EPI_FC2>(g, status, st);
-    case EPI_MERGE: return launch_mode<EPI_MERGE>(g, status, st);
+    case EPI_QKV:   return launch_mode<EPI_QKV>(g, g.status, st);
+    case EPI_PROJ:  return launch_mode<EPI_PROJ>(g, g.status, st);
+    case EPI_FC1:   return launch_mode<EPI_FC1>(g, g.status, st);
+    case EPI_FC2:   return launch_mode<EPI_FC2>(g, g.status, st);
+    case EPI_MERGE: return launch_mode<EPI_MERGE>(g, g.status, st);
   }
   return false;
 }
 
-}  // namespace mixaq
-
-namespace mixaq {
-bool launch_gemm(const GemmArgs& g, cudaStream_t st) { return launch_gemm_tc(g, g.status, st); }
 }  // namespace mixaq

@@ -81,7 +81,7 @@ struct AttnBranch {
   int32_t* tap_pv;           // nullable
 };
 struct AttnArgs {
-  const float* relbias;      // [heads][49][49]
+  const float* relbias;      // [heads][4][7][32][4], accumulator-fragment order
   int C, heads, shift, Hp, Wp, nwx, nW;
   AttnBranch br[2];
 };

@@ -128,7 +128,7 @@ Prepared carve_prepared(const mixaq_block_params* p, void* base) {
   const int N[4] = {3 * p->dim, p->dim, p->hidden, p->dim};
   for (int l = 0; l < 4; ++l)
     for (int b = 0; b < 2; ++b) { r.mult[l][b] = c.take<float>(N[l]); r.zc[l][b] = c.take<int32_t>(N[l]); }
-  r.relbias = c.take<float>((size_t)p->heads * WT * WT);
+  r.relbias = c.take<float>((size_t)p->heads * 4 * 7 * 32 * 4);   // fragment order, see k_prepare_relbias
   r.bytes = c.off;
   return r;
 }

@@ -5,40 +5,59 @@
 
 namespace mixaq {
 
-template <int NPL>
+// R rows per warp are in flight together: their loads are issued before any of the reductions starts.
+template <int NPL, int R>
 __global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo) {
   const int C = NPL * 32;
-  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  int lane = threadIdx.x & 31;
-  if (row >= hi.M + lo.M) return;
-  const bool is_hi = row < hi.M;
-  const LnBranch& br = is_hi ? hi : lo;
-  int m = is_hi ? row : row - hi.M;
-  long srow = m;
-  if (br.rowsrc) srow = br.rowsrc[m];
-  uint32_t code[NPL];
-  if (srow < 0) {
-    // pad token: zero after the normalisation, i.e. the code of 0.0
-    AQ q = br.q;
-    uint32_t z = quant_code(0.0f, q);
+  const int lane = threadIdx.x & 31;
+  const int total = hi.M + lo.M;
+  const int row_base = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * R;
+  if (row_base >= total) return;
+  float x[R][NPL];
+  long srow[R];
 #pragma unroll
-    for (int i = 0; i < NPL; ++i) code[i] = z;
-  } else {
-    const float* src = br.src + srow * C;
-    float x[NPL];
-#pragma unroll
-    for (int i = 0; i < NPL; ++i) x[i] = __ldg(src + lane + 32 * i);
-    float mean, rstd;
-    ln_stats<NPL>(x, (float)C, mean, rstd);
-    AQ q = br.q;
-#pragma unroll
-    for (int i = 0; i < NPL; ++i) {
-      int c = lane + 32 * i;
-      code[i] = quant_code(ln_apply(x[i], mean, rstd, __ldg(br.gamma + c), __ldg(br.beta + c)), q);
+  for (int r = 0; r < R; ++r) {
+    const int row = row_base + r;
+    srow[r] = -1;
+    if (row < total) {
+      const bool is_hi = row < hi.M;
+      const LnBranch& br = is_hi ? hi : lo;
+      const int m = is_hi ? row : row - hi.M;
+      srow[r] = br.rowsrc ? (long)br.rowsrc[m] : (long)m;
     }
   }
-  int bits = br.q.bits;
-  store_codes_lane_strided<NPL>(br.out + (long)m * (C * bits / 8), code, bits, lane);
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int row = row_base + r;
+    const float* src = (row < hi.M ? hi.src : lo.src) + (srow[r] < 0 ? 0 : srow[r]) * C;
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) x[r][i] = srow[r] < 0 ? 0.0f : __ldg(src + lane + 32 * i);
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int row = row_base + r;
+    if (row >= total) break;
+    const bool is_hi = row < hi.M;
+    const LnBranch& br = is_hi ? hi : lo;
+    const int m = is_hi ? row : row - hi.M;
+    const AQ q = br.q;
+    uint32_t code[NPL];
+    if (srow[r] < 0) {
+      // pad token: zero after the normalisation, i.e. the code of 0.0
+      const uint32_t z = quant_code(0.0f, q);
+#pragma unroll
+      for (int i = 0; i < NPL; ++i) code[i] = z;
+    } else {
+      float mean, rstd;
+      ln_stats<NPL>(x[r], (float)C, mean, rstd);
+#pragma unroll
+      for (int i = 0; i < NPL; ++i) {
+        const int c = lane + 32 * i;
+        code[i] = quant_code(ln_apply(x[r][i], mean, rstd, __ldg(br.gamma + c), __ldg(br.beta + c)), q);
+      }
+    }
+    store_codes_lane_strided<NPL>(br.out + (long)m * (C * q.bits / 8), code, q.bits, lane);
+  }
 }
 
 // patch merging: token (b, y2, x2) of the output gathers (2y2+dy, 2x2+dx) for (dy,dx) = (0,0),(1,0),(0,1),(1,1)
@@ -85,16 +104,14 @@ __global__ void __launch_bounds__(256) k_copy_rows(const float* __restrict__ x, 
 }
 
 #define MIXAQ_NPL_CASE(n, KERNEL, ...) case n: KERNEL<n><<<grid, 256, 0, st>>>(__VA_ARGS__); break;
+#define MIXAQ_LN_CASE(n, r) case n: k_ln_quant<n, r><<<(rows + 8 * r - 1) / (8 * r), 256, 0, st>>>(hi, lo); break;
 
 void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st) {
   int rows = hi.M + lo.M;
   if (rows == 0) return;
-  unsigned grid = (rows + 7) / 8;
   switch (C / 32) {
-    MIXAQ_NPL_CASE(1, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(2, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(3, k_ln_quant, hi, lo)
-    MIXAQ_NPL_CASE(4, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(6, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(8, k_ln_quant, hi, lo)
-    MIXAQ_NPL_CASE(12, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(16, k_ln_quant, hi, lo) MIXAQ_NPL_CASE(24, k_ln_quant, hi, lo)
-    MIXAQ_NPL_CASE(32, k_ln_quant, hi, lo)
+    MIXAQ_LN_CASE(1, 4) MIXAQ_LN_CASE(2, 4) MIXAQ_LN_CASE(3, 4) MIXAQ_LN_CASE(4, 4) MIXAQ_LN_CASE(6, 4)
+    MIXAQ_LN_CASE(8, 2) MIXAQ_LN_CASE(12, 2) MIXAQ_LN_CASE(16, 2) MIXAQ_LN_CASE(24, 1) MIXAQ_LN_CASE(32, 1)
     default: return;   // rejected by the host API before any launch
   }
   ++g_launches;

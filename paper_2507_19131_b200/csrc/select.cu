@@ -51,31 +51,39 @@ __global__ void __launch_bounds__(256) k_window_score(SelectArgs a) {
 }
 
 // Rank by counting: rank(w) = #{v : v precedes w in (score desc, index asc)}; ranks are a permutation.
-// The thread that owns window w also writes the batch bookkeeping of its slot.
-__global__ void __launch_bounds__(128) k_rank_emit(SelectArgs a) {
+// One warp per window: the lanes split the windows to compare against, the counts are summed over the warp,
+// and the lanes then write the batch bookkeeping of the window's slot (49 source-token indices) together.
+constexpr int RANK_WARPS = 8;
+__global__ void __launch_bounds__(RANK_WARPS * 32) k_rank_emit(SelectArgs a) {
   extern __shared__ long long s_score[];
-  int b = blockIdx.y;
+  const int b = blockIdx.y;
   const int64_t* sc = a.score + (long)b * a.nW;
   for (int i = threadIdx.x; i < a.nW; i += blockDim.x) s_score[i] = sc[i];
   __syncthreads();
-  int w = blockIdx.x * blockDim.x + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const int w = blockIdx.x * RANK_WARPS + (threadIdx.x >> 5);
   if (w >= a.nW) return;
-  long long mine = s_score[w];
-  int rank = 0;
+  const long long mine = s_score[w];
+  int cnt = 0;
   if (!a.reverse) {
-    for (int v = 0; v < a.nW; ++v) { long long o = s_score[v]; rank += (o > mine) || (o == mine && v < w); }
+    for (int v = lane; v < a.nW; v += 32) { long long o = s_score[v]; cnt += (o > mine) || (o == mine && v < w); }
   } else {
-    for (int v = 0; v < a.nW; ++v) { long long o = s_score[v]; rank += (o < mine) || (o == mine && v < w); }
+    for (int v = lane; v < a.nW; v += 32) { long long o = s_score[v]; cnt += (o < mine) || (o == mine && v < w); }
   }
-  a.order[(long)b * a.nW + rank] = w;
-  int c = rank < a.n_hi ? 0 : (rank < a.n_hi + a.n_lo ? 1 : 2);
-  a.cls[(long)b * a.nW + w] = (uint8_t)c;
-  int Hp = (a.H + WS - 1) / WS * WS, Wp = (a.W + WS - 1) / WS * WS;
+  const int rank = __reduce_add_sync(0xffffffffu, cnt);
+  const int c = rank < a.n_hi ? 0 : (rank < a.n_hi + a.n_lo ? 1 : 2);
+  const int Hp = (a.H + WS - 1) / WS * WS, Wp = (a.W + WS - 1) / WS * WS;
   int32_t* dst; long slot;
-  if (c == 0)      { slot = (long)b * a.n_hi + rank;                   dst = a.rowsrc_hi; a.win_hi[slot] = w; }
-  else if (c == 1) { slot = (long)b * a.n_lo + (rank - a.n_hi);        dst = a.rowsrc_lo; a.win_lo[slot] = w; }
+  if (c == 0)      { slot = (long)b * a.n_hi + rank;                     dst = a.rowsrc_hi; }
+  else if (c == 1) { slot = (long)b * a.n_lo + (rank - a.n_hi);          dst = a.rowsrc_lo; }
   else             { slot = (long)b * a.n_pr + (rank - a.n_hi - a.n_lo); dst = a.rowsrc_pr; }
-  for (int t = 0; t < WT; ++t) dst[slot * WT + t] = window_src(b, a.H, a.W, Hp, Wp, a.shift, a.nwx, w, t);
+  if (lane == 0) {
+    a.order[(long)b * a.nW + rank] = w;
+    a.cls[(long)b * a.nW + w] = (uint8_t)c;
+    if (c == 0) a.win_hi[slot] = w;
+    else if (c == 1) a.win_lo[slot] = w;
+  }
+  for (int t = lane; t < WT; t += 32) dst[slot * WT + t] = window_src(b, a.H, a.W, Hp, Wp, a.shift, a.nwx, w, t);
 }
 
 void launch_energy(const float* x, int32_t* energy, long ntok, int C, float inv_scale, cudaStream_t st) {
@@ -88,8 +96,8 @@ void launch_select(const SelectArgs& a, cudaStream_t st) {
   int nwin = a.B * a.nW;
   k_window_score<<<(nwin + 7) / 8, 256, 0, st>>>(a);
   ++g_launches;
-  dim3 grid((a.nW + 127) / 128, a.B);
-  k_rank_emit<<<grid, 128, (size_t)a.nW * sizeof(long long), st>>>(a);
+  dim3 grid((a.nW + RANK_WARPS - 1) / RANK_WARPS, a.B);
+  k_rank_emit<<<grid, RANK_WARPS * 32, (size_t)a.nW * sizeof(long long), st>>>(a);
   ++g_launches;
 }
 
