@@ -158,6 +158,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = load_peaks()
+    # a real (capturable) stream: on it the library replays each forward as one CUDA graph
+    torch.cuda.set_stream(torch.cuda.Stream())
     ctx = mq.Context(local)
     K, Wm = args.steps, max(args.warmup, 3)
 

@@ -179,6 +179,15 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
                                     const float* low_ratio_per_pair, const float* prune_ratio_per_pair /* nullable */,
                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* mixaq_backbone_forward replays a CUDA graph when it is called again with exactly the same arguments (same
+ * parameter structs byte for byte, pointers, sizes, ratios, workspace and stream): the first such call captures the
+ * launches on `cuda_stream`, later calls cost one graph launch on the host.  The data behind the pointers may
+ * change freely between calls.  Captured graphs are kept per context (16 at most) until mixaq_destroy.  Caching
+ * needs a stream that can be captured: calls on the legacy default stream (NULL), calls made while the caller is
+ * capturing the stream itself, and calls between mixaq_profile_begin/end launch their kernels directly.
+ * enabled = 0 switches the cache off and drops the stored graphs; it is on by default. */
+mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled);
+
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 

@@ -21,7 +21,7 @@ EXPORTS = [
     "mixaq_merge_prepare", "mixaq_stage_energy", "mixaq_block_workspace_bytes", "mixaq_block_forward",
     "mixaq_merge_workspace_bytes", "mixaq_merge_forward", "mixaq_backbone_workspace_bytes",
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
-    "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static",
+    "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -141,6 +141,9 @@ class Context:
 
     def device_status(self) -> int:
         return lib().mixaq_last_device_status(self.h, _stream_ptr())
+
+    def set_graph_cache(self, enabled: bool):
+        self.check(lib().mixaq_set_graph_cache(self.h, 1 if enabled else 0), "set_graph_cache")
 
     def launch_count(self) -> int:
         return lib().mixaq_last_launch_count(self.h)

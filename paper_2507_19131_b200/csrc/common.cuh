@@ -69,10 +69,11 @@ __device__ __forceinline__ uint32_t pack_const(int zp, int bits) {
   for (int sh = 0; sh < 32; sh += bits) r += k << sh;
   return r;
 }
-// 32 consecutive codes of one row, given as magic patterns, packed and stored (dst is 32*bits/8-byte aligned).
-template <int BITS>
-__device__ __forceinline__ void store_magic_32(uint8_t* dst, const uint32_t (&m)[32], uint32_t kpack) {
-  constexpr int PER = 32 / BITS, WORDS = BITS;   // codes per word, words per 32 codes
+// NC (16 or 32) consecutive codes of one row, given as magic patterns, packed and stored with one or two vector
+// stores (dst is NC*BITS/8-byte aligned).
+template <int BITS, int NC>
+__device__ __forceinline__ void store_magic(uint8_t* dst, const uint32_t (&m)[NC], uint32_t kpack) {
+  constexpr int PER = 32 / BITS, WORDS = NC / PER;   // codes per word, words
   uint32_t w[WORDS];
 #pragma unroll
   for (int i = 0; i < WORDS; ++i) {
@@ -81,13 +82,15 @@ __device__ __forceinline__ void store_magic_32(uint8_t* dst, const uint32_t (&m)
     for (int e = 0; e < PER; ++e) v += m[PER * i + e] << (BITS * e);
     w[i] = v;
   }
-  if (BITS == 8) {
+  if (WORDS == 8) {
     reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
     reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4 % WORDS], w[5 % WORDS], w[6 % WORDS], w[7 % WORDS]);
-  } else if (BITS == 4) {
-    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+  } else if (WORDS == 4) {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1 % WORDS], w[2 % WORDS], w[3 % WORDS]);
+  } else if (WORDS == 2) {
+    reinterpret_cast<uint2*>(dst)[0] = make_uint2(w[0], w[1 % WORDS]);
   } else {
-    reinterpret_cast<uint2*>(dst)[0] = make_uint2(w[0], w[1]);
+    reinterpret_cast<uint32_t*>(dst)[0] = w[0];
   }
 }
 
@@ -99,18 +102,46 @@ __device__ __forceinline__ float warp_sum_butterfly(float v) {
   return v;
 }
 
-// LayerNorm statistics of one row held as NPL values per lane (lane l holds channels l, l+32, ...).
+// LayerNorm statistics of R rows, each held as NPL values per lane (lane l holds channels l, l+32, ...).
+// The sums follow the contract (per-lane partial sums in channel order, then the butterfly); the divisions and the
+// square root, which are expensive instruction sequences, run once for all R rows: lane r serves row r and the
+// results are broadcast.
+template <int NPL, int R>
+__device__ __forceinline__ void ln_stats_rows(const float (&x)[R][NPL], float fC, float (&mean)[R], float (&rstd)[R]) {
+  const int lane = threadIdx.x & 31;
+  float tot = 0.0f;
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) s = __fadd_rn(s, x[r][i]);
+    s = warp_sum_butterfly(s);
+    if (lane == r) tot = s;
+  }
+  const float mean_l = __fdiv_rn(tot, fC);
+#pragma unroll
+  for (int r = 0; r < R; ++r) mean[r] = __shfl_sync(0xffffffffu, mean_l, r);
+  float vt = 0.0f;
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    float v = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) { float d = __fsub_rn(x[r][i], mean[r]); v = __fmaf_rn(d, d, v); }
+    v = warp_sum_butterfly(v);
+    if (lane == r) vt = v;
+  }
+  const float var_l = __fdiv_rn(vt, fC);
+  const float rstd_l = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var_l, 1e-5f)));
+#pragma unroll
+  for (int r = 0; r < R; ++r) rstd[r] = __shfl_sync(0xffffffffu, rstd_l, r);
+}
 template <int NPL>
 __device__ __forceinline__ void ln_stats(const float (&x)[NPL], float fC, float& mean, float& rstd) {
-  float s = 0.0f;
+  float xs[1][NPL], m[1], r[1];
 #pragma unroll
-  for (int i = 0; i < NPL; ++i) s = __fadd_rn(s, x[i]);
-  mean = __fdiv_rn(warp_sum_butterfly(s), fC);
-  float v = 0.0f;
-#pragma unroll
-  for (int i = 0; i < NPL; ++i) { float d = __fsub_rn(x[i], mean); v = __fmaf_rn(d, d, v); }
-  float var = __fdiv_rn(warp_sum_butterfly(v), fC);
-  rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, 1e-5f)));
+  for (int i = 0; i < NPL; ++i) xs[0][i] = x[i];
+  ln_stats_rows<NPL, 1>(xs, fC, m, r);
+  mean = m[0]; rstd = r[0];
 }
 
 __device__ __forceinline__ float ln_apply(float x, float mean, float rstd, float g, float b) {

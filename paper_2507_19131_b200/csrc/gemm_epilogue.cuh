@@ -1,33 +1,43 @@
 // Fused epilogues of the integer GEMMs (MixA-Q Section 3.2: shared integer weights, per-branch step sizes,
-// zero points and biases).  One call handles 32 consecutive output columns of 32 consecutive rows: the shape a
-// warp receives from a 32-lane x 32-column TMEM load (one row per thread).
+// zero points and biases).  One epilogue warp owns 32 rows (one TMEM lane quarter, one row per thread) and a
+// contiguous range of the tile's columns, which it walks in chunks of 16 columns:
 //   acc_raw[n] = sum_k a[m][k] * w[n][k]   with UNSIGNED activation codes a;
 //   acc[n]     = acc_raw[n] - z_a * sum_k w[n][k]                (zero-point correction, exact in int32)
 //   v[n]       = fma((float)acc[n], s_a*s_w[n], bias[n])
-// The per-column constants (zc, mult, bias) of the tile sit in shared memory; every lane of a warp reads the
-// same column, so the reads are broadcasts.
+// The per-column constants (zc, mult, bias) of the warp's columns sit in shared memory; every lane reads the same
+// column, so the reads are broadcasts.
 #pragma once
 #include "kernels.h"
 
 namespace mixaq {
 
-constexpr int EPI_STAGE_LD = 36;                       // floats per row of a warp's 32 x 32 staging tile (padded)
-constexpr int EPI_STAGE_FLOATS = 32 * EPI_STAGE_LD;
+constexpr int EPI_NC = 16;                             // columns per chunk
+constexpr int EPI_STAGE_FLOATS = 32 * EPI_NC;          // per-warp transposition tile of the binary32 epilogues
 
-struct ColConsts {                                     // shared-memory arrays indexed by the tile's local column
+struct ColConsts {                                     // shared-memory arrays indexed by the warp's local column
   const int32_t* zc; const float* mult; const float* bias;
 };
 
-// row0: first row of the warp's 32-row slab (global row index in the branch's matrix); lane owns row0 + lane.
-// n0: global first column of the group; lc0: its column inside the tile (index into the shared constants).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// zero-point correction + dequantization of one chunk; lc0 = first column of the chunk in the warp's constants
 template <int MODE>
-__device__ __forceinline__ void epilogue_row32(const GemmBranch& br, int N, int C, long row0, int lane, int n0, int lc0,
-                                               const ColConsts& cc, const int32_t (&acc_raw)[32], float* stage) {
-  const long m = row0 + lane;
-  const bool row_ok = m < br.M;
-  float v[32];
+__device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, bool row_ok, int n0, int lc0,
+                                          const ColConsts& cc, const int32_t (&acc_raw)[16], float (&v)[16]) {
+  if (br.tap_acc && row_ok) {
 #pragma unroll
-  for (int i4 = 0; i4 < 8; ++i4) {
+    for (int i = 0; i < EPI_NC; ++i) br.tap_acc[m * N + n0 + i] = acc_raw[i] - cc.zc[lc0 + i];
+  }
+#pragma unroll
+  for (int i4 = 0; i4 < EPI_NC / 4; ++i4) {
     const int4 z4 = *reinterpret_cast<const int4*>(cc.zc + lc0 + 4 * i4);
     const float4 m4 = *reinterpret_cast<const float4*>(cc.mult + lc0 + 4 * i4);
     const int zz[4] = {z4.x, z4.y, z4.z, z4.w};
@@ -40,64 +50,109 @@ __device__ __forceinline__ void epilogue_row32(const GemmBranch& br, int N, int 
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int i = 4 * i4 + j;
-      const int32_t acc = acc_raw[i] - zz[j];
-      if (br.tap_acc && row_ok) br.tap_acc[m * N + n0 + i] = acc;
-      const float f = __int2float_rn(acc);
+      const float f = __int2float_rn(acc_raw[i] - zz[j]);
       if (MODE == EPI_MERGE) v[i] = __fmul_rn(f, mm[j]);
       else                   v[i] = __fmaf_rn(f, mm[j], bb[j]);
     }
   }
+}
+
+// The warp's part of one output tile.  taddr: TMEM address of (the warp's lane quarter, its first column);
+// n_first: global index of that column; n_cols: how many columns the warp owns (a multiple of 16);
+// acc_ready(): waits (bounded) for the tile's accumulator, false when the CTA is giving up.
+template <int MODE, class WaitFn>
+__device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, int C, long row0, int lane, int n_first,
+                                                   int n_cols, const ColConsts& cc, uint32_t taddr, float* stage,
+                                                   WaitFn acc_ready) {
+  const long m = row0 + lane;
+  const bool row_ok = m < br.M;
+  const int n_chunks = n_cols / EPI_NC;
+
   if (MODE == EPI_QKV || MODE == EPI_FC1) {
-    AQ q = br.q0;
-    if (MODE == EPI_QKV) { int sec = n0 / C; if (sec == 1) q = br.q1; else if (sec == 2) q = br.q2; }
-    uint32_t c[32];
+    // ---- code outputs: every thread quantizes and packs the 16 codes of its own row ----
+    if (!acc_ready()) return false;
+    const int bits = br.out_bits;
+    uint8_t* out_row = br.out_codes + m * ((long)N * bits / 8);
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      const int n0 = n_first + ch * EPI_NC;
+      int32_t acc[EPI_NC];
+      tmem_ld16(taddr + (uint32_t)(ch * EPI_NC), acc);
+      float v[EPI_NC];
+      dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
+      AQ q = br.q0;
+      if (MODE == EPI_QKV) { const int sec = n0 / C; if (sec == 1) q = br.q1; else if (sec == 2) q = br.q2; }
+      uint32_t c[EPI_NC];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) c[i] = quant_magic(MODE == EPI_FC1 ? gelu_f(v[i]) : v[i], q);
-    if (row_ok) {
-      const int bits = br.out_bits;
-      uint8_t* dst = br.out_codes + m * ((long)N * bits / 8) + (long)n0 * bits / 8;
-      const uint32_t kp = pack_const(q.zp, bits);
-      if (bits == 8) store_magic_32<8>(dst, c, kp);
-      else if (bits == 4) store_magic_32<4>(dst, c, kp);
-      else store_magic_32<2>(dst, c, kp);
+      for (int i = 0; i < EPI_NC; ++i) c[i] = quant_magic(MODE == EPI_FC1 ? gelu_f(v[i]) : v[i], q);
+      if (row_ok) {
+        uint8_t* dst = out_row + (long)n0 * bits / 8;
+        const uint32_t kp = pack_const(q.zp, bits);
+        if (bits == 8) store_magic<8, EPI_NC>(dst, c, kp);
+        else if (bits == 4) store_magic<4, EPI_NC>(dst, c, kp);
+        else store_magic<2, EPI_NC>(dst, c, kp);
+      }
     }
-    return;
+    return true;
   }
-  // binary32 outputs: transpose the warp's 32 x 32 block through shared memory so that every global access
-  // is a run of full 128-byte lines (8 lanes per row) instead of 32 row-strided 16-byte pieces.
-  __syncwarp();
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-    *reinterpret_cast<float4*>(stage + lane * EPI_STAGE_LD + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+
+  // ---- binary32 outputs (proj: x1 = x_window + out; fc2: y = x1 + out scattered to the token's own position;
+  //      merge: out).  Each chunk is transposed through shared memory so that global accesses are 64-byte runs
+  //      (4 lanes per row, 8 rows per instruction).  The residual of chunk ch+1 is fetched while chunk ch is
+  //      computed; the residual of chunk 0 is fetched before the accumulator is even complete. ----
+  const int cj = lane & 3, rsub = lane >> 2;
   long src_mine = -1;
   if (MODE != EPI_MERGE && row_ok) src_mine = br.rowsrc[m];
-  __syncwarp();
-  const int cj = lane & 7, rsub = lane >> 3;
+  long res_row[4], dst_row[4];            // row offsets (in elements) of the residual and of the output, -1: none
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = 4 * i + rsub;
+  for (int i = 0; i < 4; ++i) {
+    const int r = 8 * i + rsub;
     const long mr = row0 + r;
     const long s = __shfl_sync(0xffffffffu, src_mine, r);
-    const float4 a = *reinterpret_cast<const float4*>(stage + r * EPI_STAGE_LD + 4 * cj);
-    if (mr >= br.M) continue;
-    const int col = n0 + 4 * cj;
-    if (MODE == EPI_PROJ) {
-      // x1 = x_window + out; a pad token's residual input is zero
-      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (s >= 0) x = __ldg(reinterpret_cast<const float4*>(br.res + s * N + col));
-      *reinterpret_cast<float4*>(br.out_f + mr * N + col) =
-          make_float4(__fadd_rn(x.x, a.x), __fadd_rn(x.y, a.y), __fadd_rn(x.z, a.z), __fadd_rn(x.w, a.w));
-    } else if (MODE == EPI_FC2) {
-      // y = x1 + out, written at the token's own position of the un-shifted map; pad tokens are dropped
-      if (s >= 0) {
-        const float4 x = __ldg(reinterpret_cast<const float4*>(br.res + mr * N + col));
-        *reinterpret_cast<float4*>(br.out_f + s * N + col) =
-            make_float4(__fadd_rn(x.x, a.x), __fadd_rn(x.y, a.y), __fadd_rn(x.z, a.z), __fadd_rn(x.w, a.w));
-      }
-    } else {  // EPI_MERGE
-      *reinterpret_cast<float4*>(br.out_f + mr * N + col) = a;
-    }
+    const bool ok = mr < br.M;
+    if (MODE == EPI_PROJ)     { res_row[i] = (ok && s >= 0) ? s * N : -1;  dst_row[i] = ok ? mr * N : -1; }
+    else if (MODE == EPI_FC2) { res_row[i] = (ok && s >= 0) ? mr * N : -1; dst_row[i] = (ok && s >= 0) ? s * N : -1; }
+    else                      { res_row[i] = -1;                            dst_row[i] = ok ? mr * N : -1; }
   }
+  float4 res[4], res_next[4];
+  auto fetch = [&](int ch, float4 (&dst)[4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);       // a pad token's residual input is zero
+      if (MODE != EPI_MERGE && res_row[i] >= 0)
+        dst[i] = __ldg(reinterpret_cast<const float4*>(br.res + res_row[i] + n_first + ch * EPI_NC + 4 * cj));
+    }
+  };
+  fetch(0, res);
+  if (!acc_ready()) return false;
+  for (int ch = 0; ch < n_chunks; ++ch) {
+    const int n0 = n_first + ch * EPI_NC;
+    int32_t acc[EPI_NC];
+    tmem_ld16(taddr + (uint32_t)(ch * EPI_NC), acc);
+    float v[EPI_NC];
+    dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
+    if (ch + 1 < n_chunks) fetch(ch + 1, res_next);
+    // row `lane`, logical 16-byte piece j is stored at piece j ^ ((lane >> 1) & 3): conflict-free both ways
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      *reinterpret_cast<float4*>(stage + lane * EPI_NC + 4 * (j ^ ((lane >> 1) & 3))) =
+          make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = 8 * i + rsub;
+      const float4 a = *reinterpret_cast<const float4*>(stage + r * EPI_NC + 4 * (cj ^ ((r >> 1) & 3)));
+      if (dst_row[i] >= 0) {
+        float4 o;
+        if (MODE == EPI_MERGE) o = a;
+        else o = make_float4(__fadd_rn(res[i].x, a.x), __fadd_rn(res[i].y, a.y), __fadd_rn(res[i].z, a.z), __fadd_rn(res[i].w, a.w));
+        *reinterpret_cast<float4*>(br.out_f + dst_row[i] + n0 + 4 * cj) = o;
+      }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) res[i] = res_next[i];
+  }
+  return true;
 }
 
 }  // namespace mixaq

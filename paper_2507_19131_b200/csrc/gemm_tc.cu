@@ -12,7 +12,7 @@
 //               staging slot of the stage; these warps expand them to one code per byte, shared to shared, into
 //               the swizzled layout (rows whose byte pitch is no multiple of 16 cannot be described to the TMA
 //               unit and are read with plain loads instead);
-//   warps 4-11  epilogue: tcgen05.ld (one row per thread, 32 columns per load) + the fused epilogue of the mode.
+//   warps 4-11  epilogue: tcgen05.ld (one row per thread, 16 columns per load) + the fused epilogue of the mode.
 // Every wait on an mbarrier is bounded; on expiry the CTA raises the status word, drains, frees its tensor
 // memory and returns.
 #include <cuda.h>
@@ -31,7 +31,7 @@ constexpr int NUM_UNPACK_WARPS = 2;            // warps 2..3
 constexpr int NUM_UNPACK_THREADS = NUM_UNPACK_WARPS * 32;
 constexpr int NUM_EPI_WARPS = 8;               // warps 4..11
 constexpr int MAX_BN = 256;
-constexpr int EPI_WARP_COLS = MAX_BN / 2;      // columns one epilogue warp handles per tile (every other 32-group)
+constexpr int EPI_WARP_COLS = MAX_BN / 2;      // columns one epilogue warp handles per tile (one half of the tile)
 constexpr int MAX_RING = 6;
 constexpr uint32_t MAX_POLLS = 1u << 22;
 constexpr int UNPACK_ITEMS = BM * (BK / UMMA_K) / NUM_UNPACK_THREADS;   // (row, 32-code group) items per thread and stage
@@ -54,7 +54,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_b
   L.stage_bytes = A_STAGE_BYTES + BN * BK + packed_bytes;
   L.ring_bytes = ring * L.stage_bytes;
   L.consts_off = L.ring_bytes;                                  // per epilogue warp (zc, mult, bias) x 128 columns
-  L.stage_off = L.consts_off + NUM_EPI_WARPS * 3 * EPI_WARP_COLS * 4;   // per epilogue warp 32 x 36 floats
+  L.stage_off = L.consts_off + NUM_EPI_WARPS * 3 * EPI_WARP_COLS * 4;   // per epilogue warp 32 x 16 floats
   L.bars_off = L.stage_off + NUM_EPI_WARPS * EPI_STAGE_FLOATS * 4;
   L.total = L.bars_off + (3 * MAX_RING + 4) * 8 + 16;
   return L;
@@ -117,19 +117,6 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
 struct TileCoord { int mt, nt; bool is_hi; };
 __device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int t) {
   TileCoord c;
@@ -294,37 +281,37 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     }
     __syncwarp();
   } else {
-    // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).., column groups e/4, e/4+2, ... ----
+    // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).. and owns half e/4 of the tile's columns ----
     const int e = warp - 4, q = warp & 3, half = e >> 2;
     float* stage = s_stage + e * EPI_STAGE_FLOATS;
     int32_t* c_zc = s_consts + e * 3 * EPI_WARP_COLS;
     float* c_mult = reinterpret_cast<float*>(c_zc + EPI_WARP_COLS);
     float* c_bias = c_mult + EPI_WARP_COLS;
+    const int n_cols = p.BN >> 1;                              // BN is a multiple of 32
     int lt = 0;
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++lt) {
       const TileCoord tc = decode_tile(p, t);
       const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
       const int a = lt & 1;
-      const int n0 = tc.nt * p.BN;
-      // per-column constants of this warp's column groups, in the warp's own shared-memory slot
+      const int n_first = tc.nt * p.BN + half * n_cols;
+      // per-column constants of this warp's columns, in the warp's own shared-memory slot
       // (no CTA-wide barrier: the only waits of this kernel are the bounded mbarrier waits)
       __syncwarp();
-      for (int grp = half, j = 0; grp < p.BN / 32; grp += 2, ++j) {
-        const int n = n0 + grp * 32 + lane;
-        c_zc[j * 32 + lane] = __ldg(br.zc + n);
-        c_mult[j * 32 + lane] = __ldg(br.mult + n);
-        if (MODE != EPI_MERGE) c_bias[j * 32 + lane] = __ldg(br.bias + n);
+      for (int j = lane; j < n_cols; j += 32) {
+        c_zc[j] = __ldg(br.zc + n_first + j);
+        c_mult[j] = __ldg(br.mult + n_first + j);
+        if (MODE != EPI_MERGE) c_bias[j] = __ldg(br.bias + n_first + j);
       }
       __syncwarp();
-      if (!mbar_wait(bar_tfull + 8u * a, (lt >> 1) & 1, abort_flag)) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       ColConsts cc; cc.zc = c_zc; cc.mult = c_mult; cc.bias = c_bias;
       const long row0 = (long)tc.mt * BM + q * 32;
-      for (int grp = half, j = 0; grp < p.BN / 32; grp += 2, ++j) {
-        int32_t acc[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_stride + grp * 32), acc);
-        epilogue_row32<MODE>(br, p.g.N, p.g.C, row0, lane, n0 + grp * 32, j * 32, cc, acc, stage);
-      }
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_stride + half * n_cols);
+      auto acc_ready = [&]() -> bool {
+        if (!mbar_wait(bar_tfull + 8u * a, (lt >> 1) & 1, abort_flag)) return false;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        return true;
+      };
+      if (!epilogue_warp_tile<MODE>(br, p.g.N, p.g.C, row0, lane, n_first, n_cols, cc, taddr, stage, acc_ready)) break;
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * a);
@@ -444,11 +431,6 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   }
   if (!make_map(&mB, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN)) return false;
   const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes).total + 1024 /*alignment slack*/;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(k_gemm_tc<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    attr_set = true;
-  }
   const int grid = p.total_tiles < sms ? p.total_tiles : sms;
   k_gemm_tc<MODE><<<grid, NUM_THREADS, smem, st>>>(mA[0], mA[1], mB, p);
   ++g_launches;
@@ -456,6 +438,18 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
 }
 
 }  // namespace
+
+// One-time set-up per device context (kept out of the launch path so that launches can be stream-captured):
+// opt-in to large dynamic shared memory for every epilogue mode, resolve the tensor-map encoder, read the SM count.
+bool gemm_init() {
+  bool ok = encode_fn() != nullptr && num_sms() > 0;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  return ok;
+}
 
 bool launch_gemm(const GemmArgs& g, cudaStream_t st) {
   switch (g.mode) {

@@ -23,7 +23,8 @@ struct SelectArgs {
   int32_t* win_lo;           // [B*n_lo]
   int B, H, W, shift, nwx, nW, n_hi, n_lo, n_pr, reverse;
 };
-void launch_select(const SelectArgs& a, cudaStream_t st);   // 2 launches
+// selections of `count` blocks that share one energy map (all blocks of a stage): 2 launches per 24 blocks
+void launch_select(const SelectArgs* a, int count, cudaStream_t st);
 
 // ---- row-wise LayerNorm + quantize + pack -----------------------------------------------------
 struct LnBranch {
@@ -67,6 +68,7 @@ struct GemmArgs {
   GemmBranch br[2];
 };
 bool launch_gemm(const GemmArgs& g, cudaStream_t st);
+bool gemm_init();   // once per device context, before the first launch
 
 // ---- fused window attention ----------------------------------------------------------------------
 struct AttnBranch {

@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <string>
 #include <vector>
 
 namespace mixaq {
@@ -18,12 +19,16 @@ int g_launches = 0;
 using namespace mixaq;
 
 struct ProfRec { int cat; cudaEvent_t e0, e1; };
+// One captured backbone forward: the exact bytes of every argument that shaped it, and the instantiated graph.
+struct GraphEntry { std::string key; cudaGraphExec_t exec; int launches; };
 struct mixaq_ctx {
   int device;
   int* d_status;
   int launches;
   char err[256];
   bool profiling;
+  bool graph_cache;                    // replay backbone forwards as CUDA graphs (see mixaq_set_graph_cache)
+  std::vector<GraphEntry> graphs;
   std::vector<ProfRec> prof;          // event pairs recorded since mixaq_profile_begin
   std::vector<cudaEvent_t> pool;      // events ready for reuse
 };
@@ -144,10 +149,24 @@ Geometry geometry(int H, int W, float low, float prune) {
   return g;
 }
 
+// buffers the selection kernels fill for one block (all sized for the worst split)
+struct SelWs {
+  int64_t* score; int32_t* order; uint8_t* cls; int32_t *rowsrc[3], *win[2]; size_t bytes;
+};
+SelWs carve_sel(int B, int H, int W, void* base) {
+  SelWs w; Carver c(base);
+  Geometry g = geometry(H, W, 0.f, 0.f);
+  const size_t slots = (size_t)B * g.nW, rows = slots * WT;
+  w.score = c.take<int64_t>(slots); w.order = c.take<int32_t>(slots); w.cls = c.take<uint8_t>(slots);
+  for (int i = 0; i < 3; ++i) w.rowsrc[i] = c.take<int32_t>(rows);
+  for (int i = 0; i < 2; ++i) w.win[i] = c.take<int32_t>(slots);
+  w.bytes = c.off;
+  return w;
+}
+
 // workspace of one block call; sized for the worst split (all windows in the wider branch)
 struct BlockWs {
-  int32_t* energy; int64_t* score; int32_t* order; uint8_t* cls;
-  int32_t *rowsrc[3], *win[2];
+  int32_t* energy; SelWs sel;
   uint8_t *a[2], *qkv[2], *o[2], *f1[2], *f2[2]; float* x1[2];
   size_t bytes;
 };
@@ -157,9 +176,8 @@ BlockWs carve_block(const mixaq_block_params* p, int B, int H, int W, void* base
   const size_t slots = (size_t)B * g.nW, rows = slots * WT;
   const int C = p->dim, Hd = p->hidden;
   w.energy = c.take<int32_t>((size_t)B * H * W);
-  w.score = c.take<int64_t>(slots); w.order = c.take<int32_t>(slots); w.cls = c.take<uint8_t>(slots);
-  for (int i = 0; i < 3; ++i) w.rowsrc[i] = c.take<int32_t>(rows);
-  for (int i = 0; i < 2; ++i) w.win[i] = c.take<int32_t>(slots);
+  w.sel = carve_sel(B, H, W, base ? (char*)base + c.off : nullptr);
+  c.off += w.sel.bytes;
   for (int i = 0; i < 2; ++i) {
     const int bits = i == 0 ? p->hi.bits : p->lo.bits;
     w.a[i]   = c.take<uint8_t>(rows * C * bits / 8);
@@ -171,6 +189,17 @@ BlockWs carve_block(const mixaq_block_params* p, int B, int H, int W, void* base
   }
   w.bytes = c.off;
   return w;
+}
+
+SelectArgs make_select_args(const SelWs& sel, const int32_t* energy, int B, int H, int W, int shift, const Geometry& g,
+                            int reverse) {
+  SelectArgs sa;
+  sa.energy = energy; sa.score = sel.score; sa.order = sel.order; sa.cls = sel.cls;
+  sa.rowsrc_hi = sel.rowsrc[0]; sa.rowsrc_lo = sel.rowsrc[1]; sa.rowsrc_pr = sel.rowsrc[2];
+  sa.win_hi = sel.win[0]; sa.win_lo = sel.win[1];
+  sa.B = B; sa.H = H; sa.W = W; sa.shift = shift; sa.nwx = g.nwx; sa.nW = g.nW;
+  sa.n_hi = g.n_hi; sa.n_lo = g.n_lo; sa.n_pr = g.n_pr; sa.reverse = reverse;
+  return sa;
 }
 
 void fill_gemm_branch(GemmBranch& g, const uint8_t* a, int M, int a_bits, const float* mult, const int32_t* zc,
@@ -202,9 +231,10 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false;
-  if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) {
-    cudaGetLastError(); delete c; return MIXAQ_CUDA_ERROR;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true;
+  if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
+      !gemm_init()) {
+    cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
   }
   *out = c;
   return MIXAQ_OK;
@@ -213,6 +243,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
 mixaq_status mixaq_destroy(mixaq_ctx* ctx) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   if (ctx->d_status) cudaFree(ctx->d_status);
+  for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& r : ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
   for (auto e : ctx->pool) cudaEventDestroy(e);
   delete ctx;
@@ -311,11 +342,14 @@ size_t mixaq_block_workspace_bytes(const mixaq_block_params* p, int B, int H, in
   return carve_block(p, B, H, W, nullptr).bytes;
 }
 
-mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, const float* x, float* y,
-                                 int B, int H, int W, float low_ratio, float prune_ratio,
-                                 const mixaq_select_opts* opts, const mixaq_selection* sel_out,
-                                 void* workspace, size_t workspace_bytes, const mixaq_taps* taps,
-                                 void* cuda_stream) {
+}  // extern "C"
+
+// `presel`: selection buffers already filled for this block (the backbone selects once per stage); NULL: select here.
+static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params* p, const float* x, float* y,
+                                       int B, int H, int W, float low_ratio, float prune_ratio,
+                                       const mixaq_select_opts* opts, const mixaq_selection* sel_out,
+                                       void* workspace, size_t workspace_bytes, const mixaq_taps* taps,
+                                       const SelWs* presel, void* cuda_stream) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   mixaq_status s = validate_block(ctx, p);
   if (s != MIXAQ_OK) return s;
@@ -336,20 +370,18 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
   g_launches = 0;
 
   // 1. scores and selection
-  const int32_t* energy = opts ? opts->energy : nullptr;
-  if (!energy) { PROF(PC_ENERGY); launch_energy(x, ws.energy, (long)B * H * W, C, p->score_inv_scale, st); energy = ws.energy; }
-  SelectArgs sa;
-  sa.energy = energy; sa.score = ws.score; sa.order = ws.order; sa.cls = ws.cls;
-  sa.rowsrc_hi = ws.rowsrc[0]; sa.rowsrc_lo = ws.rowsrc[1]; sa.rowsrc_pr = ws.rowsrc[2];
-  sa.win_hi = ws.win[0]; sa.win_lo = ws.win[1];
-  sa.B = B; sa.H = H; sa.W = W; sa.shift = p->shift; sa.nwx = g.nwx; sa.nW = g.nW;
-  sa.n_hi = g.n_hi; sa.n_lo = g.n_lo; sa.n_pr = g.n_pr; sa.reverse = opts ? opts->reverse : 0;
-  { PROF(PC_SELECT); launch_select(sa, st); }
+  const SelWs& sel = presel ? *presel : ws.sel;
+  if (!presel) {
+    const int32_t* energy = opts ? opts->energy : nullptr;
+    if (!energy) { PROF(PC_ENERGY); launch_energy(x, ws.energy, (long)B * H * W, C, p->score_inv_scale, st); energy = ws.energy; }
+    SelectArgs sa = make_select_args(sel, energy, B, H, W, p->shift, g, opts ? opts->reverse : 0);
+    { PROF(PC_SELECT); launch_select(&sa, 1, st); }
+  }
   if (sel_out) {
     const size_t n = (size_t)B * g.nW;
-    if (sel_out->cls)   cudaMemcpyAsync(sel_out->cls, ws.cls, n, cudaMemcpyDeviceToDevice, st);
-    if (sel_out->order) cudaMemcpyAsync(sel_out->order, ws.order, n * 4, cudaMemcpyDeviceToDevice, st);
-    if (sel_out->score) cudaMemcpyAsync(sel_out->score, ws.score, n * 8, cudaMemcpyDeviceToDevice, st);
+    if (sel_out->cls)   cudaMemcpyAsync(sel_out->cls, sel.cls, n, cudaMemcpyDeviceToDevice, st);
+    if (sel_out->order) cudaMemcpyAsync(sel_out->order, sel.order, n * 4, cudaMemcpyDeviceToDevice, st);
+    if (sel_out->score) cudaMemcpyAsync(sel_out->score, sel.score, n * 8, cudaMemcpyDeviceToDevice, st);
   }
 
   const mixaq_branch* brp[2] = {&p->hi, &p->lo};
@@ -360,7 +392,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
   // 2. gather + LN1 + quantize + pack
   LnBranch lb[2];
   for (int i = 0; i < 2; ++i) {
-    lb[i].src = x; lb[i].rowsrc = ws.rowsrc[i]; lb[i].gamma = brp[i]->ln1_g; lb[i].beta = brp[i]->ln1_b;
+    lb[i].src = x; lb[i].rowsrc = sel.rowsrc[i]; lb[i].gamma = brp[i]->ln1_g; lb[i].beta = brp[i]->ln1_b;
     lb[i].out = ws.a[i]; lb[i].q = to_aq(brp[i]->qkv_in); lb[i].M = M[i];
   }
   { PROF(PC_LN1); launch_ln_quant(lb[0], lb[1], C, st); }
@@ -384,7 +416,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
   const float rs = (float)(1.0 / std::sqrt((double)HEAD_DIM));
   for (int i = 0; i < 2; ++i) {
     AttnBranch& ab = aa.br[i];
-    ab.qkv = ws.qkv[i]; ab.out = ws.o[i]; ab.win = ws.win[i];
+    ab.qkv = ws.qkv[i]; ab.out = ws.o[i]; ab.win = sel.win[i];
     ab.q = to_aq(brp[i]->q); ab.k = to_aq(brp[i]->k); ab.v = to_aq(brp[i]->v); ab.o = to_aq(brp[i]->proj_in);
     ab.bits = brp[i]->bits; ab.slots = slots[i];
     ab.alpha = (brp[i]->q.scale * brp[i]->k.scale) * rs;
@@ -397,7 +429,7 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
   ga.w = p->proj.codes; ga.N = C; ga.K = C; ga.mode = EPI_PROJ;
   for (int i = 0; i < 2; ++i) {
     fill_gemm_branch(ga.br[i], ws.o[i], M[i], brp[i]->bits, pr.mult[1][i], pr.zc[1][i], brp[i]->b_proj);
-    ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = ws.rowsrc[i];
+    ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = sel.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->proj_acc : nullptr;
   }
   { PROF(PC_PROJ); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
@@ -422,13 +454,13 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
   ga.w = p->fc2.codes; ga.N = C; ga.K = Hd; ga.mode = EPI_FC2;
   for (int i = 0; i < 2; ++i) {
     fill_gemm_branch(ga.br[i], ws.f2[i], M[i], brp[i]->bits, pr.mult[3][i], pr.zc[3][i], brp[i]->b_fc2);
-    ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = ws.rowsrc[i];
+    ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = sel.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc2_acc : nullptr;
   }
   { PROF(PC_FC2); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 9. pruned windows are forwarded unchanged
-  { PROF(PC_COPY); launch_copy_rows(x, y, ws.rowsrc[2], B * g.n_pr * WT, C, st); }
+  if (g.n_pr > 0) { PROF(PC_COPY); launch_copy_rows(x, y, sel.rowsrc[2], B * g.n_pr * WT, C, st); }
 
   if (taps) {
     for (int i = 0; i < 2; ++i) {
@@ -444,6 +476,17 @@ mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, co
   }
   ctx->launches = g_launches;
   return check_cuda(ctx, "block_forward");
+}
+
+extern "C" {
+
+mixaq_status mixaq_block_forward(mixaq_ctx* ctx, const mixaq_block_params* p, const float* x, float* y,
+                                 int B, int H, int W, float low_ratio, float prune_ratio,
+                                 const mixaq_select_opts* opts, const mixaq_selection* sel_out,
+                                 void* workspace, size_t workspace_bytes, const mixaq_taps* taps,
+                                 void* cuda_stream) {
+  return block_forward_impl(ctx, p, x, y, B, H, W, low_ratio, prune_ratio, opts, sel_out, workspace, workspace_bytes,
+                            taps, nullptr, cuda_stream);
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -486,10 +529,10 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
 
 // -------------------------------------------------------------------------------------------------
 namespace {
-struct BackboneWs { float* scratch; int32_t* energy; void* merge; void* block; size_t merge_bytes, block_bytes, bytes; };
+struct BackboneWs { float* scratch; int32_t* energy; void* merge; void* block; char* sel; size_t merge_bytes, block_bytes, sel_bytes, bytes; };
 BackboneWs carve_backbone(const mixaq_backbone_params* p, int B, int H0, int W0, void* base) {
   BackboneWs w; Carver c(base);
-  size_t max_map = 0, max_tok = 0, max_merge = 0, max_block = 0;
+  size_t max_map = 0, max_tok = 0, max_merge = 0, max_block = 0, max_sel = 0;
   int H = H0, W = W0, blk = 0;
   for (int s = 0; s < p->num_stages; ++s) {
     if (s > 0) {
@@ -501,11 +544,13 @@ BackboneWs carve_backbone(const mixaq_backbone_params* p, int B, int H0, int W0,
     max_tok = std::max(max_tok, (size_t)B * H * W);
     for (int i = 0; i < p->depths[s]; ++i, ++blk)
       max_block = std::max(max_block, mixaq_block_workspace_bytes(&p->blocks[blk], B, H, W));
+    max_sel = std::max(max_sel, (size_t)p->depths[s] * carve_sel(B, H, W, nullptr).bytes);   // one set per block of the stage
   }
   w.scratch = c.take<float>(max_map);
   w.energy = c.take<int32_t>(max_tok);
   w.merge = c.take<uint8_t>(max_merge); w.merge_bytes = align_up(max_merge);
   w.block = c.take<uint8_t>(max_block); w.block_bytes = align_up(max_block);
+  w.sel = (char*)c.take<uint8_t>(max_sel); w.sel_bytes = align_up(max_sel);
   w.bytes = c.off;
   return w;
 }
@@ -541,35 +586,107 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   BackboneWs ws = carve_backbone(p, B, H0, W0, workspace);
   if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "backbone workspace too small");
   cudaStream_t st = (cudaStream_t)cuda_stream;
+
+  // Replay as a CUDA graph when an identical call was captured before.  The key is the exact bytes of everything
+  // that shapes the launches: the HOST parameter structs, ratios, pointers, sizes and the stream.
+  bool use_graph = ctx->graph_cache && !ctx->profiling && st != nullptr && st != cudaStreamLegacy;
+  if (use_graph) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) { cudaGetLastError(); use_graph = false; }
+  }
+  std::string key;
+  if (use_graph) {
+    auto put = [&key](const void* ptr, size_t n) { key.append((const char*)ptr, n); };
+    const int npairs = (nblk + 1) / 2;
+    put(&p->num_stages, sizeof(int)); put(p->depths, sizeof(int) * p->num_stages);
+    put(p->blocks, sizeof(mixaq_block_params) * nblk);
+    if (p->num_stages > 1) put(p->merges, sizeof(mixaq_merge_params) * (p->num_stages - 1));
+    put(&x0, sizeof(x0)); put(stage_out, sizeof(float*) * p->num_stages);
+    const int dims[3] = {B, H0, W0}; put(dims, sizeof(dims));
+    put(low_ratio_per_pair, sizeof(float) * npairs);
+    const char has_prune = prune_ratio_per_pair ? 1 : 0; put(&has_prune, 1);
+    if (prune_ratio_per_pair) put(prune_ratio_per_pair, sizeof(float) * npairs);
+    put(&workspace, sizeof(workspace)); put(&workspace_bytes, sizeof(workspace_bytes)); put(&st, sizeof(st));
+    for (auto& g : ctx->graphs)
+      if (g.key == key) {
+        if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return check_cuda(ctx, "backbone_forward (graph launch)");
+        ctx->launches = g.launches;
+        return MIXAQ_OK;
+      }
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); use_graph = false; }
+  }
+
+  mixaq_status result = MIXAQ_OK;
   int total = 0, H = H0, W = W0, blk = 0;
   const float* cur = x0;
-  for (int s = 0; s < p->num_stages; ++s) {
+  for (int s = 0; s < p->num_stages && result == MIXAQ_OK; ++s) {
     const int d = p->depths[s];
     float* out_s = stage_out[s];
     if (s > 0) {
       // the merge writes where the first block of the stage does NOT write
       float* mdst = (d % 2 == 0) ? out_s : ws.scratch;
-      mixaq_status r = mixaq_merge_forward(ctx, &p->merges[s - 1], cur, mdst, B, H, W, ws.merge, ws.merge_bytes, st);
-      if (r != MIXAQ_OK) return r;
+      result = mixaq_merge_forward(ctx, &p->merges[s - 1], cur, mdst, B, H, W, ws.merge, ws.merge_bytes, st);
+      if (result != MIXAQ_OK) break;
       total += ctx->launches;
       cur = mdst; H = (H + 1) / 2; W = (W + 1) / 2;
     }
+    // importance is scored once per stage, before its first block (Section 3.2): one energy map, and from it the
+    // window classes and batch bookkeeping of EVERY block of the stage (own shift, own pair's ratios) in one go
     const mixaq_block_params* b0 = &p->blocks[blk];
     { PROF(PC_ENERGY); launch_energy(cur, ws.energy, (long)B * H * W, b0->dim, b0->score_inv_scale, st); }
     total += 1;
-    mixaq_select_opts so; so.energy = ws.energy; so.reverse = 0;
+    const size_t sel_stride = carve_sel(B, H, W, nullptr).bytes;
+    std::vector<SelWs> sels(d);
+    std::vector<SelectArgs> sargs(d);
+    for (int i = 0; i < d; ++i) {
+      const float lr = low_ratio_per_pair[(blk + i) / 2], pr = prune_ratio_per_pair ? prune_ratio_per_pair[(blk + i) / 2] : 0.f;
+      Geometry g = geometry(H, W, lr, pr);
+      if ((size_t)g.nW * 8 > 48 * 1024) { result = fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many windows per image (max 6144)"); break; }
+      sels[i] = carve_sel(B, H, W, ws.sel + (size_t)i * sel_stride);
+      sargs[i] = make_select_args(sels[i], ws.energy, B, H, W, p->blocks[blk + i].shift, g, 0);
+    }
+    if (result != MIXAQ_OK) break;
+    g_launches = 0;
+    { PROF(PC_SELECT); launch_select(sargs.data(), d, st); }
+    total += g_launches;
     for (int i = 0; i < d; ++i, ++blk) {
       float* dst = ((d - 1 - i) % 2 == 0) ? out_s : ws.scratch;
-      mixaq_status r = mixaq_block_forward(ctx, &p->blocks[blk], cur, dst, B, H, W, low_ratio_per_pair[blk / 2],
-                                           prune_ratio_per_pair ? prune_ratio_per_pair[blk / 2] : 0.f, &so, nullptr,
-                                           ws.block, ws.block_bytes, nullptr, st);
-      if (r != MIXAQ_OK) return r;
+      result = block_forward_impl(ctx, &p->blocks[blk], cur, dst, B, H, W, low_ratio_per_pair[blk / 2],
+                                  prune_ratio_per_pair ? prune_ratio_per_pair[blk / 2] : 0.f, nullptr, nullptr,
+                                  ws.block, ws.block_bytes, nullptr, &sels[i], st);
+      if (result != MIXAQ_OK) break;
       total += ctx->launches;
       cur = dst;
     }
   }
+  if (use_graph) {
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(st, &graph);
+    if (result != MIXAQ_OK) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return result; }
+    cudaGraphExec_t exec = nullptr;
+    if (e != cudaSuccess || !graph || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
+      if (graph) cudaGraphDestroy(graph);
+      return check_cuda(ctx, "backbone_forward (graph capture)") == MIXAQ_OK
+                 ? fail(ctx, MIXAQ_CUDA_ERROR, "backbone_forward: graph capture failed") : MIXAQ_CUDA_ERROR;
+    }
+    cudaGraphDestroy(graph);
+    if (ctx->graphs.size() >= 16) { cudaGraphExecDestroy(ctx->graphs.front().exec); ctx->graphs.erase(ctx->graphs.begin()); }
+    ctx->graphs.push_back({key, exec, total});
+    if (cudaGraphLaunch(exec, st) != cudaSuccess) return check_cuda(ctx, "backbone_forward (graph launch)");
+  }
+  if (result != MIXAQ_OK) return result;
   ctx->launches = total;
   return check_cuda(ctx, "backbone_forward");
+}
+
+mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  ctx->graph_cache = enabled != 0;
+  if (!enabled) {
+    for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
+    ctx->graphs.clear();
+  }
+  return MIXAQ_OK;
 }
 
 }  // extern "C"

@@ -33,6 +33,8 @@ __global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo) {
 #pragma unroll
     for (int i = 0; i < NPL; ++i) x[r][i] = srow[r] < 0 ? 0.0f : __ldg(src + lane + 32 * i);
   }
+  float mean[R], rstd[R];
+  ln_stats_rows<NPL, R>(x, (float)C, mean, rstd);
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const int row = row_base + r;
@@ -48,12 +50,10 @@ __global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo) {
 #pragma unroll
       for (int i = 0; i < NPL; ++i) code[i] = z;
     } else {
-      float mean, rstd;
-      ln_stats<NPL>(x[r], (float)C, mean, rstd);
 #pragma unroll
       for (int i = 0; i < NPL; ++i) {
         const int c = lane + 32 * i;
-        code[i] = quant_code(ln_apply(x[r][i], mean, rstd, __ldg(br.gamma + c), __ldg(br.beta + c)), q);
+        code[i] = quant_code(ln_apply(x[r][i], mean[r], rstd[r], __ldg(br.gamma + c), __ldg(br.beta + c)), q);
       }
     }
     store_codes_lane_strided<NPL>(br.out + (long)m * (C * q.bits / 8), code, q.bits, lane);
@@ -110,8 +110,8 @@ void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t
   int rows = hi.M + lo.M;
   if (rows == 0) return;
   switch (C / 32) {
-    MIXAQ_LN_CASE(1, 4) MIXAQ_LN_CASE(2, 4) MIXAQ_LN_CASE(3, 4) MIXAQ_LN_CASE(4, 4) MIXAQ_LN_CASE(6, 4)
-    MIXAQ_LN_CASE(8, 2) MIXAQ_LN_CASE(12, 2) MIXAQ_LN_CASE(16, 2) MIXAQ_LN_CASE(24, 1) MIXAQ_LN_CASE(32, 1)
+    MIXAQ_LN_CASE(1, 8) MIXAQ_LN_CASE(2, 8) MIXAQ_LN_CASE(3, 8) MIXAQ_LN_CASE(4, 8) MIXAQ_LN_CASE(6, 4)
+    MIXAQ_LN_CASE(8, 4) MIXAQ_LN_CASE(12, 4) MIXAQ_LN_CASE(16, 2) MIXAQ_LN_CASE(24, 2) MIXAQ_LN_CASE(32, 2)
     default: return;   // rejected by the host API before any launch
   }
   ++g_launches;

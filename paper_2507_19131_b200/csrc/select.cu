@@ -4,23 +4,30 @@
 
 namespace mixaq {
 
-// One warp per token: energy = sum_c clamp(rne(x*inv), -127, 127)^2.
+// energy[token] = sum_c clamp(rne(x*inv), -127, 127)^2.  Integer sums are exact in any order, so the loads are
+// laid out for the memory system only: a group of G = 8 lanes owns one token and walks its channels with
+// 16-byte loads (C is a multiple of 32), four tokens per warp.
+__device__ __forceinline__ int score_code_sq(float v, float inv) {
+  // clamp before rounding (the bounds are integers), then round to nearest-even by the 1.5*2^23 addition
+  float t = fminf(fmaxf(__fmul_rn(v, inv), -127.0f), 127.0f);
+  int code = (int)(__float_as_uint(__fadd_rn(t, 12582912.0f)) - kMagicBits);
+  return code * code;
+}
 __global__ void __launch_bounds__(256) k_energy(const float* __restrict__ x, int32_t* __restrict__ energy,
                                                 long ntok, int C, float inv) {
-  long tok = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  int lane = threadIdx.x & 31;
-  if (tok >= ntok) return;
-  const float* row = x + tok * C;
+  const long tok = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
+  const int sub = threadIdx.x & 7;
   int e = 0;
-  for (int c = lane; c < C; c += 32) {
-    float r = rintf(__fmul_rn(__ldg(row + c), inv));
-    r = fminf(fmaxf(r, -127.0f), 127.0f);
-    int code = __float2int_rz(r);
-    e += code * code;
+  if (tok < ntok) {
+    const float4* row = reinterpret_cast<const float4*>(x + tok * C);
+    for (int c4 = sub; c4 < C / 4; c4 += 8) {
+      const float4 v = __ldg(row + c4);
+      e += score_code_sq(v.x, inv) + score_code_sq(v.y, inv) + score_code_sq(v.z, inv) + score_code_sq(v.w, inv);
+    }
   }
 #pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) e += __shfl_xor_sync(0xffffffffu, e, off);
-  if (lane == 0) energy[tok] = e;
+  for (int off = 4; off >= 1; off >>= 1) e += __shfl_xor_sync(0xffffffffu, e, off);
+  if (sub == 0 && tok < ntok) energy[tok] = e;
 }
 
 __device__ __forceinline__ int window_src(int b, int H, int W, int Hp, int Wp, int shift, int nwx, int w, int t) {
@@ -34,7 +41,11 @@ __device__ __forceinline__ int window_src(int b, int H, int W, int Hp, int Wp, i
 
 // One warp per (image, window): score = sum of the energies of the window's real tokens under this
 // block's own (possibly shifted, cyclically wrapped) partition.
-__global__ void __launch_bounds__(256) k_window_score(SelectArgs a) {
+constexpr int MAX_SELECT_BATCH = 24;
+struct SelectBatch { SelectArgs a[MAX_SELECT_BATCH]; };
+
+__global__ void __launch_bounds__(256) k_window_score(const __grid_constant__ SelectBatch batch) {
+  const SelectArgs& a = batch.a[blockIdx.y];
   int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   int lane = threadIdx.x & 31;
   if (gw >= a.B * a.nW) return;
@@ -54,8 +65,9 @@ __global__ void __launch_bounds__(256) k_window_score(SelectArgs a) {
 // One warp per window: the lanes split the windows to compare against, the counts are summed over the warp,
 // and the lanes then write the batch bookkeeping of the window's slot (49 source-token indices) together.
 constexpr int RANK_WARPS = 8;
-__global__ void __launch_bounds__(RANK_WARPS * 32) k_rank_emit(SelectArgs a) {
+__global__ void __launch_bounds__(RANK_WARPS * 32) k_rank_emit(const __grid_constant__ SelectBatch batch) {
   extern __shared__ long long s_score[];
+  const SelectArgs& a = batch.a[blockIdx.z];
   const int b = blockIdx.y;
   const int64_t* sc = a.score + (long)b * a.nW;
   for (int i = threadIdx.x; i < a.nW; i += blockDim.x) s_score[i] = sc[i];
@@ -87,18 +99,25 @@ __global__ void __launch_bounds__(RANK_WARPS * 32) k_rank_emit(SelectArgs a) {
 }
 
 void launch_energy(const float* x, int32_t* energy, long ntok, int C, float inv_scale, cudaStream_t st) {
-  int wpb = 8;
-  k_energy<<<(unsigned)((ntok + wpb - 1) / wpb), wpb * 32, 0, st>>>(x, energy, ntok, C, inv_scale);
+  k_energy<<<(unsigned)((ntok * 8 + 255) / 256), 256, 0, st>>>(x, energy, ntok, C, inv_scale);
   ++g_launches;
 }
 
-void launch_select(const SelectArgs& a, cudaStream_t st) {
-  int nwin = a.B * a.nW;
-  k_window_score<<<(nwin + 7) / 8, 256, 0, st>>>(a);
-  ++g_launches;
-  dim3 grid((a.nW + RANK_WARPS - 1) / RANK_WARPS, a.B);
-  k_rank_emit<<<grid, RANK_WARPS * 32, (size_t)a.nW * sizeof(long long), st>>>(a);
-  ++g_launches;
+void launch_select(const SelectArgs* args, int count, cudaStream_t st) {
+  // all entries share B, H, W (one stage); shift, ratios and output buffers differ
+  for (int first = 0; first < count; first += MAX_SELECT_BATCH) {
+    const int n = count - first < MAX_SELECT_BATCH ? count - first : MAX_SELECT_BATCH;
+    SelectBatch batch;
+    for (int i = 0; i < n; ++i) batch.a[i] = args[first + i];
+    for (int i = n; i < MAX_SELECT_BATCH; ++i) batch.a[i] = args[first];
+    const SelectArgs& a = args[first];
+    const int nwin = a.B * a.nW;
+    k_window_score<<<dim3((nwin + 7) / 8, n), 256, 0, st>>>(batch);
+    ++g_launches;
+    dim3 grid((a.nW + RANK_WARPS - 1) / RANK_WARPS, a.B, n);
+    k_rank_emit<<<grid, RANK_WARPS * 32, (size_t)a.nW * sizeof(long long), st>>>(batch);
+    ++g_launches;
+  }
 }
 
 }  // namespace mixaq

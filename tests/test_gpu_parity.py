@@ -149,6 +149,25 @@ def test_backbone_tiny(orc, mq, ctx, prune):
         assert np.array_equal(g.cpu().numpy(), w)
 
 
+def test_backbone_graph_replay_reads_fresh_data(orc, mq, ctx):
+    """On a capturable stream the backbone call is captured once and replayed; replays must see new input data."""
+    wl = synth.tiny_backbone(ratio=0.4, prune=0.2)
+    dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+    xs = [wl.x, np.ascontiguousarray(wl.x[:, ::-1]), (wl.x * F32(0.5)).astype(F32)]
+    xd = dev(xs[0])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i, x in enumerate(xs):                                # call 0 captures, calls 1 and 2 replay
+            xd.copy_(torch.from_numpy(x), non_blocking=False)
+            got = mq.backbone_forward(ctx, dbb, xd, wl.low_ratios, wl.prune_ratios)
+            side.synchronize()
+            want = orc.backbone_forward(wl.backbone, x, wl.low_ratios, wl.prune_ratios)
+            for g, w in zip(got, want):
+                assert np.array_equal(g.cpu().numpy(), w), f"call {i}"
+    torch.cuda.current_stream().wait_stream(side)
+
+
 def test_config2_stage1_pair_full_size(orc, mq, ctx):
     """Block pair at 200x334 (W-MSA then SW-MSA with mask), B=2, Student-t input, ratio 0.3, shared stage energy."""
     wl = synth.config2()
