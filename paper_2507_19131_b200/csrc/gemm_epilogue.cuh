@@ -18,14 +18,22 @@ struct ColConsts {                                     // shared-memory arrays i
   const int32_t* zc; const float* mult; const float* bias;
 };
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&r)[16]) {
+// Asynchronous TMEM load of 16 columns (one row per thread); the registers are valid after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, int32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Waits for every TMEM load issued so far.  The registers pass through the statement as in-out operands so that
+// no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(int32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+      :: "memory");
 }
 
 // zero-point correction + dequantization of one chunk; lc0 = first column of the chunk in the warp's constants
@@ -73,10 +81,8 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     if (!acc_ready()) return false;
     const int bits = br.out_bits;
     uint8_t* out_row = br.out_codes + m * ((long)N * bits / 8);
-    for (int ch = 0; ch < n_chunks; ++ch) {
+    auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
       const int n0 = n_first + ch * EPI_NC;
-      int32_t acc[EPI_NC];
-      tmem_ld16(taddr + (uint32_t)(ch * EPI_NC), acc);
       float v[EPI_NC];
       dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
       AQ q = br.q0;
@@ -90,6 +96,19 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
         if (bits == 8) store_magic<8, EPI_NC>(dst, c, kp);
         else if (bits == 4) store_magic<4, EPI_NC>(dst, c, kp);
         else store_magic<2, EPI_NC>(dst, c, kp);
+      }
+    };
+    // the TMEM load of the next chunk is in flight while this chunk is computed
+    int32_t acc0[EPI_NC], acc1[EPI_NC];
+    tmem_ld16_issue(taddr, acc0);
+    for (int ch = 0; ch < n_chunks; ch += 2) {
+      tmem_ld_wait(acc0);
+      if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), acc1);
+      chunk(ch, acc0);
+      if (ch + 1 < n_chunks) {
+        tmem_ld_wait(acc1);
+        if (ch + 2 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 2) * EPI_NC), acc0);
+        chunk(ch + 1, acc1);
       }
     }
     return true;
@@ -124,10 +143,8 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
   };
   fetch(0, res);
   if (!acc_ready()) return false;
-  for (int ch = 0; ch < n_chunks; ++ch) {
+  auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
     const int n0 = n_first + ch * EPI_NC;
-    int32_t acc[EPI_NC];
-    tmem_ld16(taddr + (uint32_t)(ch * EPI_NC), acc);
     float v[EPI_NC];
     dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
     if (ch + 1 < n_chunks) fetch(ch + 1, res_next);
@@ -151,6 +168,18 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     __syncwarp();
 #pragma unroll
     for (int i = 0; i < 4; ++i) res[i] = res_next[i];
+  };
+  int32_t acc0[EPI_NC], acc1[EPI_NC];
+  tmem_ld16_issue(taddr, acc0);
+  for (int ch = 0; ch < n_chunks; ch += 2) {
+    tmem_ld_wait(acc0);
+    if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), acc1);
+    chunk(ch, acc0);
+    if (ch + 1 < n_chunks) {
+      tmem_ld_wait(acc1);
+      if (ch + 2 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 2) * EPI_NC), acc0);
+      chunk(ch + 1, acc1);
+    }
   }
   return true;
 }

@@ -288,21 +288,26 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     float* c_mult = reinterpret_cast<float*>(c_zc + EPI_WARP_COLS);
     float* c_bias = c_mult + EPI_WARP_COLS;
     const int n_cols = p.BN >> 1;                              // BN is a multiple of 32
-    int lt = 0;
+    int lt = 0, consts_key = -1;
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++lt) {
       const TileCoord tc = decode_tile(p, t);
       const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
       const int a = lt & 1;
       const int n_first = tc.nt * p.BN + half * n_cols;
-      // per-column constants of this warp's columns, in the warp's own shared-memory slot
+      // per-column constants of this warp's columns, in the warp's own shared-memory slot; they depend on the
+      // branch and the column tile only, and the grid is sized so that a CTA keeps its column tile
       // (no CTA-wide barrier: the only waits of this kernel are the bounded mbarrier waits)
-      __syncwarp();
-      for (int j = lane; j < n_cols; j += 32) {
-        c_zc[j] = __ldg(br.zc + n_first + j);
-        c_mult[j] = __ldg(br.mult + n_first + j);
-        if (MODE != EPI_MERGE) c_bias[j] = __ldg(br.bias + n_first + j);
+      const int key = tc.nt * 2 + (tc.is_hi ? 1 : 0);
+      if (key != consts_key) {
+        consts_key = key;
+        __syncwarp();
+        for (int j = lane; j < n_cols; j += 32) {
+          c_zc[j] = __ldg(br.zc + n_first + j);
+          c_mult[j] = __ldg(br.mult + n_first + j);
+          if (MODE != EPI_MERGE) c_bias[j] = __ldg(br.bias + n_first + j);
+        }
+        __syncwarp();
       }
-      __syncwarp();
       ColConsts cc; cc.zc = c_zc; cc.mult = c_mult; cc.bias = c_bias;
       const long row0 = (long)tc.mt * BM + q * 32;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_stride + half * n_cols);
@@ -431,7 +436,9 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   }
   if (!make_map(&mB, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN)) return false;
   const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes).total + 1024 /*alignment slack*/;
-  const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles)
+  int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  if (grid > p.n_tiles && grid < p.total_tiles) grid -= grid % p.n_tiles;
   k_gemm_tc<MODE><<<grid, NUM_THREADS, smem, st>>>(mA[0], mA[1], mB, p);
   ++g_launches;
   return true;

@@ -6,57 +6,50 @@
 namespace mixaq {
 
 // R rows per warp are in flight together: their loads are issued before any of the reductions starts.
+// A CTA works for one branch only (the first `blocks_hi` CTAs take the high batch), so the branch's constants
+// (gamma, beta, quantizer) are fetched once per warp and no per-row selection is left in the loop.
 template <int NPL, int R>
-__global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo) {
+__global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo, int blocks_hi) {
   const int C = NPL * 32;
   const int lane = threadIdx.x & 31;
-  const int total = hi.M + lo.M;
-  const int row_base = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * R;
-  if (row_base >= total) return;
-  float x[R][NPL];
+  const bool is_hi = (int)blockIdx.x < blocks_hi;
+  const LnBranch& br = is_hi ? hi : lo;
+  const int M = br.M;
+  const int m_base = (((is_hi ? blockIdx.x : blockIdx.x - blocks_hi) * (blockDim.x >> 5)) + (threadIdx.x >> 5)) * R;
+  if (m_base >= M) return;
+  const float* __restrict__ src = br.src;
+  const int32_t* __restrict__ rowsrc = br.rowsrc;
   long srow[R];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
-    const int row = row_base + r;
+    const int m = m_base + r;
     srow[r] = -1;
-    if (row < total) {
-      const bool is_hi = row < hi.M;
-      const LnBranch& br = is_hi ? hi : lo;
-      const int m = is_hi ? row : row - hi.M;
-      srow[r] = br.rowsrc ? (long)br.rowsrc[m] : (long)m;
-    }
+    if (m < M) srow[r] = rowsrc ? (long)rowsrc[m] : (long)m;
   }
+  float x[R][NPL];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
-    const int row = row_base + r;
-    const float* src = (row < hi.M ? hi.src : lo.src) + (srow[r] < 0 ? 0 : srow[r]) * C;
+    const float* row = src + (srow[r] < 0 ? 0 : srow[r]) * C + lane;
 #pragma unroll
-    for (int i = 0; i < NPL; ++i) x[r][i] = srow[r] < 0 ? 0.0f : __ldg(src + lane + 32 * i);
+    for (int i = 0; i < NPL; ++i) x[r][i] = srow[r] < 0 ? 0.0f : __ldg(row + 32 * i);
   }
+  float gam[NPL], bet[NPL];
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) { gam[i] = __ldg(br.gamma + lane + 32 * i); bet[i] = __ldg(br.beta + lane + 32 * i); }
+  const AQ q = br.q;
+  const int row_bytes = C * q.bits / 8;
   float mean[R], rstd[R];
   ln_stats_rows<NPL, R>(x, (float)C, mean, rstd);
+  const uint32_t zcode = quant_code(0.0f, q);      // pad token: zero after the normalisation
 #pragma unroll
   for (int r = 0; r < R; ++r) {
-    const int row = row_base + r;
-    if (row >= total) break;
-    const bool is_hi = row < hi.M;
-    const LnBranch& br = is_hi ? hi : lo;
-    const int m = is_hi ? row : row - hi.M;
-    const AQ q = br.q;
+    const int m = m_base + r;
+    if (m >= M) break;
     uint32_t code[NPL];
-    if (srow[r] < 0) {
-      // pad token: zero after the normalisation, i.e. the code of 0.0
-      const uint32_t z = quant_code(0.0f, q);
 #pragma unroll
-      for (int i = 0; i < NPL; ++i) code[i] = z;
-    } else {
-#pragma unroll
-      for (int i = 0; i < NPL; ++i) {
-        const int c = lane + 32 * i;
-        code[i] = quant_code(ln_apply(x[r][i], mean[r], rstd[r], __ldg(br.gamma + c), __ldg(br.beta + c)), q);
-      }
-    }
-    store_codes_lane_strided<NPL>(br.out + (long)m * (C * q.bits / 8), code, q.bits, lane);
+    for (int i = 0; i < NPL; ++i)
+      code[i] = srow[r] < 0 ? zcode : quant_code(ln_apply(x[r][i], mean[r], rstd[r], gam[i], bet[i]), q);
+    store_codes_lane_strided<NPL>(br.out + (long)m * row_bytes, code, q.bits, lane);
   }
 }
 
@@ -104,14 +97,29 @@ __global__ void __launch_bounds__(256) k_copy_rows(const float* __restrict__ x, 
 }
 
 #define MIXAQ_NPL_CASE(n, KERNEL, ...) case n: KERNEL<n><<<grid, 256, 0, st>>>(__VA_ARGS__); break;
-#define MIXAQ_LN_CASE(n, r) case n: k_ln_quant<n, r><<<(rows + 8 * r - 1) / (8 * r), 256, 0, st>>>(hi, lo); break;
+template <int NPL, int R>
+void launch_ln_r(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
+  const int rows_per_block = 8 * R;
+  const int bh = (hi.M + rows_per_block - 1) / rows_per_block, bl = (lo.M + rows_per_block - 1) / rows_per_block;
+  k_ln_quant<NPL, R><<<bh + bl, 256, 0, st>>>(hi, lo, bh);
+}
+// rows per warp: more rows amortise the per-warp constants and the divisions, but small problems need the warps
+template <int NPL, int RMAX>
+void launch_ln_npl(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
+  const int rows = hi.M + lo.M;
+  if (RMAX >= 8 && rows >= 8 * 8 * 148 * 4) launch_ln_r<NPL, (RMAX >= 8 ? 8 : RMAX)>(hi, lo, st);
+  else if (RMAX >= 4 && rows >= 4 * 8 * 148 * 4) launch_ln_r<NPL, (RMAX >= 4 ? 4 : RMAX)>(hi, lo, st);
+  else if (RMAX >= 2 && rows >= 2 * 8 * 148 * 4) launch_ln_r<NPL, (RMAX >= 2 ? 2 : RMAX)>(hi, lo, st);
+  else launch_ln_r<NPL, 1>(hi, lo, st);
+}
+#define MIXAQ_NPL_CASE(n, KERNEL, ...) case n: KERNEL<n><<<grid, 256, 0, st>>>(__VA_ARGS__); break;
+#define MIXAQ_LN_CASE(n, rmax) case n: launch_ln_npl<n, rmax>(hi, lo, st); break;
 
 void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st) {
-  int rows = hi.M + lo.M;
-  if (rows == 0) return;
+  if (hi.M + lo.M == 0) return;
   switch (C / 32) {
     MIXAQ_LN_CASE(1, 8) MIXAQ_LN_CASE(2, 8) MIXAQ_LN_CASE(3, 8) MIXAQ_LN_CASE(4, 8) MIXAQ_LN_CASE(6, 4)
-    MIXAQ_LN_CASE(8, 4) MIXAQ_LN_CASE(12, 4) MIXAQ_LN_CASE(16, 2) MIXAQ_LN_CASE(24, 2) MIXAQ_LN_CASE(32, 2)
+    MIXAQ_LN_CASE(8, 4) MIXAQ_LN_CASE(12, 2) MIXAQ_LN_CASE(16, 2) MIXAQ_LN_CASE(24, 1) MIXAQ_LN_CASE(32, 1)
     default: return;   // rejected by the host API before any launch
   }
   ++g_launches;
