@@ -132,6 +132,7 @@ def algorithmic_work(wl, mq):
                 add("gemm_proj", ops=2.0 * M * C * C, byt=M * (C * cb + C * 4 + C * 4))
                 add("ln2_quant", byt=M * (C * 4 + C * cb))
                 add("gemm_fc1_gelu", ops=2.0 * M * C * Hd, byt=M * (C * cb + Hd * cb))
+                work["gemm_fc1_gelu"]["alu_ops"] = work["gemm_fc1_gelu"].get("alu_ops", 0.0) + FC1_EPILOGUE_OPS * M * Hd
                 add("gemm_fc2_scatter", ops=2.0 * M * Hd * C, byt=M * (Hd * cb + C * 4 + C * 4))
             add("select", byt=B * H * W * 4)
             add("copy_pruned", byt=B * n_pr * 49 * C * 8)
@@ -139,9 +140,18 @@ def algorithmic_work(wl, mq):
     return work
 
 
+# The fc1 epilogue (zero-point correction, dequantize, GELU, quantize, pack) is a fixed sequence of binary32 / integer
+# lane operations per output, set by the numeric contract: 3 (int subtract, convert, fma) + 20 (GELU: |v| clamp, 7 fma,
+# 3 adds of the rounding split, 5 fma, exponent insert, multiply, max, subtract) + 4 (quantize) + 1 (pack) = 28.
+# With K = C <= 768 the MMA needs K/64 <= 12 clocks per output row-chunk where the epilogue needs 28 issue slots, so
+# the kernel is bound by plain ALU issue; its peak is SMs x 128 lanes x SM clock.
+FC1_EPILOGUE_OPS = 28
+ALU_CATS = {"gemm_fc1_gelu"}
+NUM_SMS, LANES_PER_SM = 148, 128
 TENSOR_CATS = {"gemm_qkv", "gemm_proj", "gemm_fc1_gelu", "gemm_fc2_scatter", "gemm_merge"}
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None
-NCU_TRAFFIC_PER_LAUNCH = {}
+# (stage-1 launch of the category, the largest of its 12 launches per step; profiles/gemm_tc_stage1_ncu_full.md)
+NCU_TRAFFIC_PER_LAUNCH = {"gemm_fc1_gelu": 5.03e6, "gemm_fc2_scatter": 47.5e6, "gemm_qkv": 5.02e6, "gemm_proj": 31.2e6}
 
 
 def run_ours(args):
@@ -236,7 +246,15 @@ def run_ours(args):
         v["share"] = round(v["ms_per_step"] / tot, 4)
     dom = max(kernels, key=lambda c: kernels[c]["ms_per_step"])
     dk = kernels[dom]
-    if dom in TENSOR_CATS:
+    if dom in ALU_CATS:
+        clk = (main["clocks"] or {}).get("sm_mhz") or 1965.0
+        peak = NUM_SMS * LANES_PER_SM * clk * 1e6 / 1e12          # T lane-ops/s at the SM clock sampled under load
+        ach = work[dom]["alu_ops"] / (dk["ms_per_step"] * 1e-3) / 1e12
+        roof = dict(kernel=dom, bound="alu", achieved=round(ach, 3), peak=round(peak, 3), unit="T lane-op/s",
+                    frac=round(ach / peak, 5),
+                    peak_source="148 SMs x 128 lanes x sampled SM clock; 28 contract operations per fc1 output",
+                    tensor_tops=dk["tops"], tensor_frac=round(dk["tops"] / (2.0 * peaks["bf16_sustained"]), 5))
+    elif dom in TENSOR_CATS:
         peak = 2.0 * peaks["bf16_sustained"]      # int8 dense = 2 x bf16 (nominal ratio) on the measured bf16 peak
         roof = dict(kernel=dom, bound="tensor", achieved=dk["tops"], peak=peak, unit="TOP/s(int8)",
                     frac=round(dk["tops"] / peak, 5),
@@ -247,6 +265,7 @@ def run_ours(args):
                     frac=round(dk["gbs"] / peak, 5), peak_source=f"hbm_gbs of {peaks['source']} peaks")
     roof["launch_us"] = round(1e3 * dk["ms_per_step"] / max(1, dk["launches_per_step"]), 3)
     roof["traffic"] = NCU_TRAFFIC_PER_LAUNCH.get(dom)
+    roof["traffic_note"] = "dram bytes of the category's stage-1 launch (ncu); activations are largely L2-resident"
     roof["timed"] = "separate pass of K steps with CUDA events around every kernel, on the launching stream"
 
     # end to end through the public call with HOST buffers (pinned): H2D of the image, forward, D2H of the 4 maps

@@ -99,17 +99,16 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
       }
     };
     // the TMEM load of the next chunk is in flight while this chunk is computed
-    int32_t acc0[EPI_NC], acc1[EPI_NC];
-    tmem_ld16_issue(taddr, acc0);
-    for (int ch = 0; ch < n_chunks; ch += 2) {
-      tmem_ld_wait(acc0);
-      if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), acc1);
-      chunk(ch, acc0);
-      if (ch + 1 < n_chunks) {
-        tmem_ld_wait(acc1);
-        if (ch + 2 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 2) * EPI_NC), acc0);
-        chunk(ch + 1, acc1);
-      }
+    // (one copy of the chunk body keeps the loop inside the instruction cache: the prefetched registers are moved)
+    int32_t acc[EPI_NC], nxt[EPI_NC];
+    tmem_ld16_issue(taddr, nxt);
+#pragma unroll 1
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      tmem_ld_wait(nxt);
+#pragma unroll
+      for (int i = 0; i < EPI_NC; ++i) acc[i] = nxt[i];
+      if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), nxt);
+      chunk(ch, acc);
     }
     return true;
   }
@@ -169,17 +168,15 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
 #pragma unroll
     for (int i = 0; i < 4; ++i) res[i] = res_next[i];
   };
-  int32_t acc0[EPI_NC], acc1[EPI_NC];
-  tmem_ld16_issue(taddr, acc0);
-  for (int ch = 0; ch < n_chunks; ch += 2) {
-    tmem_ld_wait(acc0);
-    if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), acc1);
-    chunk(ch, acc0);
-    if (ch + 1 < n_chunks) {
-      tmem_ld_wait(acc1);
-      if (ch + 2 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 2) * EPI_NC), acc0);
-      chunk(ch + 1, acc1);
-    }
+  int32_t acc[EPI_NC], nxt[EPI_NC];
+  tmem_ld16_issue(taddr, nxt);
+#pragma unroll 1
+  for (int ch = 0; ch < n_chunks; ++ch) {
+    tmem_ld_wait(nxt);
+#pragma unroll
+    for (int i = 0; i < EPI_NC; ++i) acc[i] = nxt[i];
+    if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), nxt);
+    chunk(ch, acc);
   }
   return true;
 }

@@ -33,7 +33,7 @@ constexpr int NUM_EPI_WARPS = 8;               // warps 4..11
 constexpr int MAX_BN = 256;
 constexpr int EPI_WARP_COLS = MAX_BN / 2;      // columns one epilogue warp handles per tile (one half of the tile)
 constexpr int MAX_RING = 6;
-constexpr uint32_t MAX_POLLS = 1u << 22;
+constexpr uint32_t MAX_POLLS = 1u << 20;       // tries per wait; each try may sleep up to WAIT_HINT_NS
 constexpr int UNPACK_ITEMS = BM * (BK / UMMA_K) / NUM_UNPACK_THREADS;   // (row, 32-code group) items per thread and stage
 
 struct TcParams {
@@ -71,20 +71,23 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One try: the thread is suspended by the hardware until the phase completes or the time hint (nanoseconds)
+// runs out, so a waiting warp does not take issue slots from the warps that work.
+constexpr uint32_t WAIT_HINT_NS = 20000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
   return ok != 0;
 }
 // Bounded wait.  Returns false when the limit ran out or another thread of the CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < MAX_POLLS; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 63u && *abort_flag) return false;
+    if (*abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
