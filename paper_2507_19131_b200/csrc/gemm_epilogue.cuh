@@ -1,6 +1,6 @@
 // Fused epilogues of the integer GEMMs (MixA-Q Section 3.2: shared integer weights, per-branch step sizes,
-// zero points and biases).  One epilogue warp owns 32 rows (one TMEM lane quarter, one row per thread) and a
-// contiguous range of the tile's columns, which it walks in chunks of 16 columns:
+// zero points and biases).  One epilogue warp owns 32 rows (one TMEM lane quarter, one row per thread) and every
+// c_step-th 16-column chunk of the tile (the warps that share a lane quarter deal the chunks round-robin):
 //   acc_raw[n] = sum_k a[m][k] * w[n][k]   with UNSIGNED activation codes a;
 //   acc[n]     = acc_raw[n] - z_a * sum_k w[n][k]                (zero-point correction, exact in int32)
 //   v[n]       = fma((float)acc[n], s_a*s_w[n], bias[n])
@@ -65,16 +65,20 @@ __device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, b
   }
 }
 
-// The warp's part of one output tile.  taddr: TMEM address of (the warp's lane quarter, its first column);
-// n_first: global index of that column; n_cols: how many columns the warp owns (a multiple of 16);
+// The warp's part of one output tile.  taddr: TMEM address of (the warp's lane quarter, the tile's first column);
+// n_tile0: global index of that column; the warp owns the tile's chunks c_first, c_first + c_step, ... < c_total
+// (its constants are stored densely: chunk number j of the warp at local column 16 j);
 // acc_ready(): waits (bounded) for the tile's accumulator, false when the CTA is giving up.
 template <int MODE, class WaitFn>
-__device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, int C, long row0, int lane, int n_first,
-                                                   int n_cols, const ColConsts& cc, uint32_t taddr, float* stage,
-                                                   WaitFn acc_ready) {
+__device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, int C, long row0, int lane, int n_tile0,
+                                                   int c_first, int c_step, int c_total, const ColConsts& cc,
+                                                   uint32_t taddr_tile, float* stage, WaitFn acc_ready) {
   const long m = row0 + lane;
   const bool row_ok = m < br.M;
-  const int n_chunks = n_cols / EPI_NC;
+  const int n_chunks = c_first < c_total ? (c_total - c_first + c_step - 1) / c_step : 0;
+  const int n_first = n_tile0 + c_first * EPI_NC;          // global column of the warp's first chunk
+  const int col_step = c_step * EPI_NC;                    // distance between consecutive chunks of the warp
+  const uint32_t taddr = taddr_tile + (uint32_t)(c_first * EPI_NC);
 
   if (MODE == EPI_QKV || MODE == EPI_FC1) {
     // ---- code outputs: every thread quantizes and packs the 16 codes of its own row ----
@@ -82,7 +86,7 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     const int bits = br.out_bits;
     uint8_t* out_row = br.out_codes + m * ((long)N * bits / 8);
     auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
-      const int n0 = n_first + ch * EPI_NC;
+      const int n0 = n_first + ch * col_step;
       float v[EPI_NC];
       dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
       AQ q = br.q0;
@@ -101,13 +105,13 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     // the TMEM load of the next chunk is in flight while this chunk is computed
     // (one copy of the chunk body keeps the loop inside the instruction cache: the prefetched registers are moved)
     int32_t acc[EPI_NC], nxt[EPI_NC];
-    tmem_ld16_issue(taddr, nxt);
+    if (n_chunks > 0) tmem_ld16_issue(taddr, nxt);
 #pragma unroll 1
     for (int ch = 0; ch < n_chunks; ++ch) {
       tmem_ld_wait(nxt);
 #pragma unroll
       for (int i = 0; i < EPI_NC; ++i) acc[i] = nxt[i];
-      if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), nxt);
+      if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * col_step), nxt);
       chunk(ch, acc);
     }
     return true;
@@ -137,13 +141,13 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     for (int i = 0; i < 4; ++i) {
       dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);       // a pad token's residual input is zero
       if (MODE != EPI_MERGE && res_row[i] >= 0)
-        dst[i] = __ldg(reinterpret_cast<const float4*>(br.res + res_row[i] + n_first + ch * EPI_NC + 4 * cj));
+        dst[i] = __ldg(reinterpret_cast<const float4*>(br.res + res_row[i] + n_first + ch * col_step + 4 * cj));
     }
   };
-  fetch(0, res);
+  if (n_chunks > 0) fetch(0, res);
   if (!acc_ready()) return false;
   auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
-    const int n0 = n_first + ch * EPI_NC;
+    const int n0 = n_first + ch * col_step;
     float v[EPI_NC];
     dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
     if (ch + 1 < n_chunks) fetch(ch + 1, res_next);
@@ -169,13 +173,13 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     for (int i = 0; i < 4; ++i) res[i] = res_next[i];
   };
   int32_t acc[EPI_NC], nxt[EPI_NC];
-  tmem_ld16_issue(taddr, nxt);
+  if (n_chunks > 0) tmem_ld16_issue(taddr, nxt);
 #pragma unroll 1
   for (int ch = 0; ch < n_chunks; ++ch) {
     tmem_ld_wait(nxt);
 #pragma unroll
     for (int i = 0; i < EPI_NC; ++i) acc[i] = nxt[i];
-    if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * EPI_NC), nxt);
+    if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * col_step), nxt);
     chunk(ch, acc);
   }
   return true;

@@ -12,7 +12,7 @@
 //               staging slot of the stage; these warps expand them to one code per byte, shared to shared, into
 //               the swizzled layout (rows whose byte pitch is no multiple of 16 cannot be described to the TMA
 //               unit and are read with plain loads instead);
-//   warps 4-11  epilogue: tcgen05.ld (one row per thread, 16 columns per load) + the fused epilogue of the mode.
+//   warps 4-..  epilogue (16 warps for the code outputs, 8 for the binary32 outputs): tcgen05.ld (one row per thread, 16 columns per load) + the fused epilogue of the mode.
 // Every wait on an mbarrier is bounded; on expiry the CTA raises the status word, drains, frees its tensor
 // memory and returns.
 #include <cuda.h>
@@ -26,12 +26,12 @@ constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int BK = 128;            // codes (bytes) per row and stage = one 128-byte swizzle row
 constexpr int UMMA_K = 32;         // codes per tcgen05.mma kind::i8
 constexpr int A_STAGE_BYTES = BM * BK;
-constexpr int NUM_THREADS = 384;
 constexpr int NUM_UNPACK_WARPS = 2;            // warps 2..3
 constexpr int NUM_UNPACK_THREADS = NUM_UNPACK_WARPS * 32;
-constexpr int NUM_EPI_WARPS = 8;               // warps 4..11
+constexpr int MAX_EPI_WARPS = 16;              // warps 4.. : 16 for the arithmetic-bound code epilogues, 8 for the binary32 ones
+__host__ __device__ constexpr int epi_warps(int mode) { return (mode == EPI_QKV || mode == EPI_FC1) ? 16 : 8; }
 constexpr int MAX_BN = 256;
-constexpr int EPI_WARP_COLS = MAX_BN / 2;      // columns one epilogue warp handles per tile (one half of the tile)
+constexpr int EPI_WARP_COLS = MAX_BN / 2;      // most columns one epilogue warp handles per tile (two warps per lane quarter)
 constexpr int MAX_RING = 6;
 constexpr uint32_t MAX_POLLS = 1u << 20;       // tries per wait; each try may sleep up to WAIT_HINT_NS
 constexpr int UNPACK_ITEMS = BM * (BK / UMMA_K) / NUM_UNPACK_THREADS;   // (row, 32-code group) items per thread and stage
@@ -50,6 +50,7 @@ struct SmemLayout {
   int stage_bytes, ring_bytes, consts_off, stage_off, bars_off, total;
 };
 __host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_bytes) {
+  constexpr int NUM_EPI_WARPS = MAX_EPI_WARPS;
   SmemLayout L;
   L.stage_bytes = A_STAGE_BYTES + BN * BK + packed_bytes;
   L.ring_bytes = ring * L.stage_bytes;
@@ -131,7 +132,7 @@ __device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int t) {
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(128 + 32 * epi_warps(MODE), 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
           const __grid_constant__ CUtensorMap tmB, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -148,10 +149,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 3 * MAX_RING + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
+  constexpr int NUM_EPI_WARPS = epi_warps(MODE);
+  constexpr int EPI_SPLIT = NUM_EPI_WARPS / 4;   // warps that share a TMEM lane quarter deal its chunks round-robin
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int K = p.g.K;
   const int acc_stride = p.tmem_cols >> 1;                     // TMEM columns between the two accumulators
 
+  if (tid == 32) {
+    // the descriptors are fetched while the barriers are set up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA0) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA1) : "memory");
+  }
   if (tid == 0) {
     for (int s = 0; s < p.ring; ++s) {
       mbar_init(bar_full + 8u * s, 1u + NUM_UNPACK_WARPS);      // TMA thread + one arrival per unpack warp
@@ -284,42 +293,46 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     }
     __syncwarp();
   } else {
-    // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).. and owns half e/4 of the tile's columns ----
-    const int e = warp - 4, q = warp & 3, half = e >> 2;
+    // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).. and takes every EPI_SPLIT-th 16-column chunk ----
+    const int e = warp - 4, q = warp & 3, sub = e >> 2;
     float* stage = s_stage + e * EPI_STAGE_FLOATS;
     int32_t* c_zc = s_consts + e * 3 * EPI_WARP_COLS;
     float* c_mult = reinterpret_cast<float*>(c_zc + EPI_WARP_COLS);
     float* c_bias = c_mult + EPI_WARP_COLS;
-    const int n_cols = p.BN >> 1;                              // BN is a multiple of 32
+    const int c_total = p.BN / EPI_NC;                         // BN is a multiple of 32
     int lt = 0, consts_key = -1;
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++lt) {
       const TileCoord tc = decode_tile(p, t);
       const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
       const int a = lt & 1;
-      const int n_first = tc.nt * p.BN + half * n_cols;
-      // per-column constants of this warp's columns, in the warp's own shared-memory slot; they depend on the
-      // branch and the column tile only, and the grid is sized so that a CTA keeps its column tile
+      const int n_tile0 = tc.nt * p.BN;
+      // per-column constants of this warp's chunks, densely in the warp's own shared-memory slot; they depend on
+      // the branch and the column tile only, and the grid is sized so that a CTA keeps its column tile
       // (no CTA-wide barrier: the only waits of this kernel are the bounded mbarrier waits)
       const int key = tc.nt * 2 + (tc.is_hi ? 1 : 0);
       if (key != consts_key) {
         consts_key = key;
         __syncwarp();
-        for (int j = lane; j < n_cols; j += 32) {
-          c_zc[j] = __ldg(br.zc + n_first + j);
-          c_mult[j] = __ldg(br.mult + n_first + j);
-          if (MODE != EPI_MERGE) c_bias[j] = __ldg(br.bias + n_first + j);
+        for (int c = sub, j = 0; c < c_total; c += EPI_SPLIT, ++j) {
+          if (lane < EPI_NC) {
+            const int n = n_tile0 + c * EPI_NC + lane;
+            c_zc[j * EPI_NC + lane] = __ldg(br.zc + n);
+            c_mult[j * EPI_NC + lane] = __ldg(br.mult + n);
+            if (MODE != EPI_MERGE) c_bias[j * EPI_NC + lane] = __ldg(br.bias + n);
+          }
         }
         __syncwarp();
       }
       ColConsts cc; cc.zc = c_zc; cc.mult = c_mult; cc.bias = c_bias;
       const long row0 = (long)tc.mt * BM + q * 32;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_stride + half * n_cols);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_stride);
       auto acc_ready = [&]() -> bool {
         if (!mbar_wait(bar_tfull + 8u * a, (lt >> 1) & 1, abort_flag)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         return true;
       };
-      if (!epilogue_warp_tile<MODE>(br, p.g.N, p.g.C, row0, lane, n_first, n_cols, cc, taddr, stage, acc_ready)) break;
+      if (!epilogue_warp_tile<MODE>(br, p.g.N, p.g.C, row0, lane, n_tile0, sub, EPI_SPLIT, c_total, cc, taddr, stage,
+                                    acc_ready)) break;
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * a);
@@ -442,7 +455,7 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles)
   int grid = p.total_tiles < sms ? p.total_tiles : sms;
   if (grid > p.n_tiles && grid < p.total_tiles) grid -= grid % p.n_tiles;
-  k_gemm_tc<MODE><<<grid, NUM_THREADS, smem, st>>>(mA[0], mA[1], mB, p);
+  k_gemm_tc<MODE><<<grid, 128 + 32 * epi_warps(MODE), smem, st>>>(mA[0], mA[1], mB, p);
   ++g_launches;
   return true;
 }
