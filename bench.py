@@ -221,6 +221,52 @@ def run_ours(args):
         d2h = sum(h.numel() * 4 for h in outs_host) if e2e else 0
         return dict(ms=ms, wall=wall, clocks=clocks, launches=launches, h2d=h2d, d2h=d2h, wl=wl, dbb=dbb, x_dev=x_dev)
 
+    def time_e2e(ratio, steps, warm):
+        wl = workload(ratio)
+        x_host = torch.from_numpy(np.roll(wl.x, rank, axis=1).copy()).pin_memory()
+        comp = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        sets = []
+        for _ in range(2):
+            dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+            sets.append(dict(dbb=dbb, x=torch.empty_like(x_host, device="cuda"),
+                             host=[torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in dbb.outs],
+                             e_in=torch.cuda.Event(), e_comp=torch.cuda.Event(), e_out=torch.cuda.Event()))
+        torch.cuda.synchronize()
+
+        def step(i):
+            b = sets[i % 2]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(b["e_comp"])                 # the forward that last read this input buffer is done
+                b["x"].copy_(x_host, non_blocking=True)
+                b["e_in"].record(s_in)
+            comp.wait_event(b["e_in"])
+            comp.wait_event(b["e_out"])                      # the previous results of this set have left the device
+            flush.fill_(i & 0xFF)
+            outs = mq.backbone_forward(ctx, b["dbb"], b["x"], wl.low_ratios, wl.prune_ratios)
+            b["e_comp"].record(comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(b["e_comp"])
+                for h, o in zip(b["host"], outs):
+                    h.copy_(o, non_blocking=True)
+                b["e_out"].record(s_out)
+
+        for i in range(warm + 2):
+            step(i)
+        barrier()
+        t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_begin.record(comp)
+        s_in.wait_event(t_begin); s_out.wait_event(t_begin)
+        for i in range(steps):
+            step(i)
+        comp.wait_stream(s_out); comp.wait_stream(s_in)
+        t_end.record(comp)
+        barrier()
+        t = torch.tensor([t_begin.elapsed_time(t_end)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return dict(ms=float(t.item()), wl=wl, h2d=x_host.numel() * 4, d2h=sum(h.numel() * 4 for h in sets[0]["host"]))
+
     sampler = ClockSampler(local) if rank == 0 else None
     main = time_ratio(args.ratio, K, Wm, sampler)
     ms_per_step = main["ms"] / K
@@ -268,8 +314,10 @@ def run_ours(args):
     roof["traffic_note"] = "dram bytes of the category's stage-1 launch (ncu); activations are largely L2-resident"
     roof["timed"] = "separate pass of K steps with CUDA events around every kernel, on the launching stream"
 
-    # end to end through the public call with HOST buffers (pinned): H2D of the image, forward, D2H of the 4 maps
-    e2e = time_ratio(args.ratio, K, Wm, None, e2e=True)
+    # end to end through the public call with HOST buffers (pinned): every step copies its image host->device, runs
+    # the forward and copies the four stage maps device->host.  Two buffer sets and three streams let the copies of
+    # neighbouring steps overlap the compute (PCIe is full duplex); the timed region is the whole pipeline of K steps.
+    e2e = time_e2e(args.ratio, K, Wm)
     e2e_value = world * wl_images(e2e["wl"]) * K / (e2e["ms"] / 1e3)
 
     sweep = {}
@@ -297,7 +345,8 @@ def run_ours(args):
                    "parallelism": "replicas only (one image per GPU, no collective)"},
         "clocks": main["clocks"],
         "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
-                "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": round(e2e["ms"] / K, 4)},
+                "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": round(e2e["ms"] / K, 4),
+                "pipeline": "2 buffer sets, copy-in / compute / copy-out streams; K steps timed as one pipeline"},
         "gpu_launches": main["launches"] * K,
         "roofline": roof,
         "kernels": kernels,

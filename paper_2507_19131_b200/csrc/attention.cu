@@ -4,7 +4,8 @@
 //   P = softmax_row(S) in binary32  ->  P codes (unsigned, step 1/(2^b-1))
 //   O_int = P_codes (v - z_v) (int32)  ->  O = O_int * s_p*s_v  ->  codes of the proj input quantizer.
 //
-// One warp per (window slot, head).  Both products run on the integer tensor cores of the warp
+// One CTA of four warps per (window slot, head): the warps stage q, k and v together, then warp i owns query rows
+// 16i .. 16i+15.  Both products run on the integer tensor cores of the warp
 // (mma.sync m16n8k32, u8 x u8 -> s32; 49 tokens padded to 64 query rows x 56 key columns).  The 49 x 32 problem is
 // far too small for a 128-row tcgen05 tile and is bound by the softmax arithmetic, not by the MMA rate.
 // The softmax runs on the accumulator fragments: a quad of lanes holds one row, lane t of the quad owns columns
@@ -27,7 +28,7 @@ struct WarpSmem {
   uint32_t vt[32][VT_LD];     // V^T: row e, 64 key positions in the permuted order of pos()
   int rq[64];                 // per query row:  -z_k * sum_d q + 32 z_q z_k
   int ck[56];                 // per key column: -z_q * sum_d k
-  uint32_t o[16][8];          // staging of 16 output rows x 32 codes (one per byte)
+  uint32_t o[4][16][8];       // per warp: staging of 16 output rows x 32 codes (one per byte)
   uint8_t reg[64];            // shift region of every token
 };
 
@@ -72,71 +73,55 @@ __device__ __forceinline__ uint32_t squeeze_pairs(uint32_t t) {
 
 template <bool SHIFTED>
 __global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
-  __shared__ __align__(16) WarpSmem smem_all[ATT_WARPS];
+  __shared__ __align__(16) WarpSmem sm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int slots_hi = a.br[0].slots;
-  const long wg = (long)blockIdx.x * ATT_WARPS + warp;
-  if (wg >= (long)(slots_hi + a.br[1].slots) * a.heads) return;
+  const long wg = (long)blockIdx.x;
   int slot = (int)(wg / a.heads);
   const int h = (int)(wg - (long)slot * a.heads);
   const bool is_hi = slot < slots_hi;
   const AttnBranch& br = is_hi ? a.br[0] : a.br[1];
   if (!is_hi) slot -= slots_hi;
-  WarpSmem& sm = smem_all[warp];
   const int bits = br.bits, C = a.C;
   const long row_bytes = (long)3 * C * bits / 8;
   const int zq = br.q.zp, zk = br.k.zp, zv = br.v.zp;
 
-  // ---- stage q, k (rows) and v (transposed, permuted) of this head, one code per byte ----
+  // ---- stage q, k (rows) and v (transposed, permuted) of this head, one code per byte: 3 x 64 row items ----
   int wy = 0, wx = 0;
   if (SHIFTED) { const int w = br.win[slot]; wy = w / a.nwx; wx = w - wy * a.nwx; }
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const int r = lane + 32 * half;
-    const int p = pos(r);
-    uint8_t* vtb = reinterpret_cast<uint8_t*>(&sm.vt[0][0]);
-    if (r < WT) {
-      const uint8_t* src = br.qkv + ((long)slot * WT + r) * row_bytes + (long)(h * HEAD_DIM) * bits / 8;
-      uint32_t w[8];
-      load_codes_32(src, bits, w);
+  for (int item = threadIdx.x; item < 3 * 64; item += ATT_WARPS * 32) {
+    const int sec = item >> 6, r = item & 63;
+    const uint8_t* src = br.qkv + ((long)slot * WT + r) * row_bytes + (long)(sec * C + h * HEAD_DIM) * bits / 8;
+    uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (r < WT) load_codes_32(src, bits, w);
+    if (sec < 2) {
       int s = 0;
 #pragma unroll
       for (int e = 0; e < 8; ++e) s = dp4a_uu(w[e], 0x01010101u, s);
-      *reinterpret_cast<uint4*>(&sm.q[r][0]) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4*>(&sm.q[r][4]) = make_uint4(w[4], w[5], w[6], w[7]);
-      sm.rq[r] = -zk * s + HEAD_DIM * zq * zk;
-      load_codes_32(src + (long)C * bits / 8, bits, w);
-      s = 0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) s = dp4a_uu(w[e], 0x01010101u, s);
-      *reinterpret_cast<uint4*>(&sm.k[r][0]) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4*>(&sm.k[r][4]) = make_uint4(w[4], w[5], w[6], w[7]);
-      sm.ck[r] = -zq * s;
-      load_codes_32(src + (long)2 * C * bits / 8, bits, w);
+      if (sec == 0) {
+        *reinterpret_cast<uint4*>(&sm.q[r][0]) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(&sm.q[r][4]) = make_uint4(w[4], w[5], w[6], w[7]);
+        sm.rq[r] = r < WT ? -zk * s + HEAD_DIM * zq * zk : 0;
+        int reg = 0;
+        if (SHIFTED && r < WT) {
+          const int i = r / WS, j = r - i * WS;
+          reg = shift_region(wy * WS + i, a.Hp, a.shift) * 3 + shift_region(wx * WS + j, a.Wp, a.shift);
+        }
+        sm.reg[r] = (uint8_t)reg;
+      } else if (r < 56) {
+        *reinterpret_cast<uint4*>(&sm.k[r][0]) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(&sm.k[r][4]) = make_uint4(w[4], w[5], w[6], w[7]);
+        sm.ck[r] = -zq * s;
+      }
+    } else {
+      uint8_t* vtb = reinterpret_cast<uint8_t*>(&sm.vt[0][0]);
+      const int p = pos(r);
 #pragma unroll
       for (int e = 0; e < 32; ++e) vtb[e * (VT_LD * 4) + p] = (uint8_t)(w[e >> 2] >> (8 * (e & 3)));
-      int reg = 0;
-      if (SHIFTED) {
-        const int i = r / WS, j = r - i * WS;
-        reg = shift_region(wy * WS + i, a.Hp, a.shift) * 3 + shift_region(wx * WS + j, a.Wp, a.shift);
-      }
-      sm.reg[r] = (uint8_t)reg;
-    } else {
-      *reinterpret_cast<uint4*>(&sm.q[r][0]) = make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4*>(&sm.q[r][4]) = make_uint4(0, 0, 0, 0);
-      sm.rq[r] = 0;
-      sm.reg[r] = 0;
-      if (r < 56) {
-        *reinterpret_cast<uint4*>(&sm.k[r][0]) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(&sm.k[r][4]) = make_uint4(0, 0, 0, 0);
-        sm.ck[r] = 0;
-      }
-#pragma unroll
-      for (int e = 0; e < 32; ++e) vtb[e * (VT_LD * 4) + p] = 0;
     }
   }
-  __syncwarp();
+  __syncthreads();
 
   // ---- key fragments, per-column terms and regions of this lane's 14 columns (fixed over the query tiles) ----
   uint32_t kb0[7], kb1[7];
@@ -165,8 +150,8 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
   const long m_base = (long)slot * WT;
   const long out_row_bytes = (long)C * bits / 8;
 
-#pragma unroll 1
-  for (int mt = 0; mt < 4; ++mt) {
+  {
+    const int mt = warp;
     // ---- S = Q K^T for 16 query rows ----
     uint32_t qa[4];
     qa[0] = sm.q[16 * mt + g][t];     qa[1] = sm.q[16 * mt + g + 8][t];
@@ -257,7 +242,6 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
       for (int ks = 0; ks < 2; ++ks)
         mma_u8(d[ne], pa[ks], sm.vt[8 * ne + g][8 * ks + t], sm.vt[8 * ne + g][8 * ks + 4 + t]);
     }
-    __syncwarp();                               // the previous tile's rows have left the staging area
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
       const int i = 16 * mt + g + 8 * r;
@@ -271,15 +255,15 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
           const uint32_t code = quant_code(__fmul_rn(__int2float_rn(o_int), so), oq);
           two |= code << (8 * u);
         }
-        reinterpret_cast<uint16_t*>(&sm.o[g + 8 * r][0])[4 * ne + t] = (uint16_t)two;
+        reinterpret_cast<uint16_t*>(&sm.o[warp][g + 8 * r][0])[4 * ne + t] = (uint16_t)two;
       }
     }
     __syncwarp();
     if (lane < 16) {
       const int i = 16 * mt + lane;
       if (i < WT) {
-        const uint4 w0 = *reinterpret_cast<const uint4*>(&sm.o[lane][0]);
-        const uint4 w1 = *reinterpret_cast<const uint4*>(&sm.o[lane][4]);
+        const uint4 w0 = *reinterpret_cast<const uint4*>(&sm.o[warp][lane][0]);
+        const uint4 w1 = *reinterpret_cast<const uint4*>(&sm.o[warp][lane][4]);
         uint8_t* dst = br.out + (m_base + i) * out_row_bytes + (long)h * HEAD_DIM * bits / 8;
         if (bits == 8) {
           reinterpret_cast<uint4*>(dst)[0] = w0;
@@ -304,7 +288,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
 void launch_attention(const AttnArgs& a, cudaStream_t st) {
   const long problems = (long)(a.br[0].slots + a.br[1].slots) * a.heads;
   if (problems == 0) return;
-  const unsigned grid = (unsigned)((problems + ATT_WARPS - 1) / ATT_WARPS);
+  const unsigned grid = (unsigned)problems;
   if (a.shift > 0) k_attention<true><<<grid, ATT_WARPS * 32, 0, st>>>(a);
   else             k_attention<false><<<grid, ATT_WARPS * 32, 0, st>>>(a);
   ++g_launches;
