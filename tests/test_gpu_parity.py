@@ -180,6 +180,41 @@ def test_config2_stage1_pair_full_size(orc, mq, ctx):
     assert np.array_equal(y, want[0])
 
 
+def _full_backbone_case(orc, mq, ctx, wl):
+    """Whole backbone at a benchmark configuration's full size, launched the way bench.py launches it (own stream, so
+    the second call replays the captured graph); every stage map against the oracle."""
+    want = orc.backbone_forward(wl.backbone, wl.x, wl.low_ratios, wl.prune_ratios)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+        xd = dev(wl.x)
+        for call in range(2):
+            got = mq.backbone_forward(ctx, dbb, xd, wl.low_ratios, wl.prune_ratios)
+            side.synchronize()
+            assert ctx.device_status() == 0
+            for st, (g, w) in enumerate(zip(got, want)):
+                g = g.cpu().numpy()
+                assert_close_rel(g, w)
+                assert np.array_equal(g, w), f"stage {st} (call {call}) within tolerance but not bit-identical"
+    torch.cuda.current_stream().wait_stream(side)
+
+
+def test_config3_swin_t_800x1333_full_size(orc, mq, ctx):
+    """Swin-T, 200x334 tokens, W4, A8/A4, ratio 0.25: the benchmark workload."""
+    _full_backbone_case(orc, mq, ctx, synth.config3(ratio=0.25))
+
+
+def test_config4_swin_s_1024_full_size_three_classes(orc, mq, ctx):
+    """Swin-S, B=4, 256x256 tokens, W4, A4 high / A2 low, ratio 0.5, 20 % of the windows pruned."""
+    _full_backbone_case(orc, mq, ctx, synth.config4())
+
+
+def test_config5_swin_b_1536_full_size(orc, mq, ctx):
+    """Swin-B, B=2, 384x384 tokens, W8, A8/A4, clustered high-norm regions, ratio 0.5."""
+    _full_backbone_case(orc, mq, ctx, synth.config5(ratio=0.5))
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
     import ctypes as C
     blk = synth.make_block(np.random.default_rng(40), 32, 1, 0, 8, 8, 4)
