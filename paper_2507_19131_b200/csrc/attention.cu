@@ -72,7 +72,7 @@ __device__ __forceinline__ uint32_t squeeze_pairs(uint32_t t) {
 }
 
 template <bool SHIFTED>
-__global__ void __launch_bounds__(ATT_WARPS * 32) k_attention(AttnArgs a) {
+__global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
   __shared__ __align__(16) WarpSmem sm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
