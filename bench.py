@@ -329,6 +329,14 @@ def run_ours(args):
             s = time_ratio(r, max(3, K // 2), 3)
             sweep[str(r)] = round(wl_images(s["wl"]) * max(3, K // 2) / (s["ms"] / 1e3), 2)
 
+    # the paper's axis: relative cost in bit operations (Appendix 6.2) of every swept ratio, with this shape's MACs
+    from paper_2507_19131_b200 import cost_model as cm
+    bbm = main["wl"].backbone
+    pair_g, fixed_g = cm.backbone_pair_gmacs(bbm.dims, bbm.depths, main["wl"].H, main["wl"].W)
+    cost = {str(r): {"relative_bops": round(cm.relative_cost([r] * len(pair_g), pair_g, fixed_g), 4),
+                     "equivalent_act_bits": round(cm.equivalent_act_bits([r] * len(pair_g), 8.0, pair_g, fixed_g), 3)}
+            for r in (SWEEP if args.sweep else [args.ratio])}
+
     status = ctx.device_status()
     if rank != 0:
         if world > 1:
@@ -351,6 +359,7 @@ def run_ours(args):
         "roofline": roof,
         "kernels": kernels,
         "low_ratio_sweep_images_per_sec": sweep,
+        "paper_cost_model": cost,
         "device_status": status,
     }
     if args.cpu_baseline and world == 1:
