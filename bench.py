@@ -89,8 +89,17 @@ class ClockSampler:
         return out
 
 
+CONFIG = 3          # --config: 3 = Swin-T 800x1333 (the metric's workload), 4 = Swin-S 1024^2 B=4, 5 = Swin-B 1536^2 B=2
+
+
 def workload(ratio: float):
     from paper_2507_19131_b200 import synth
+    if CONFIG == 4:
+        wl = synth.config4()
+        wl.low_ratios = [ratio] * len(wl.low_ratios)
+        return wl
+    if CONFIG == 5:
+        return synth.config5(ratio=ratio)
     return synth.config3(ratio=ratio)
 
 
@@ -158,6 +167,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2507_19131_b200 import binding as mq
+    from paper_2507_19131_b200 import replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -183,7 +193,7 @@ def run_ours(args):
     def time_ratio(ratio, steps, warm, sampler=None, e2e=False):
         wl = workload(ratio)
         # replicas differ only in their seed-shifted input (weak scaling: one image per rank per step)
-        x_host = torch.from_numpy(np.roll(wl.x, rank, axis=1).copy()).pin_memory()
+        x_host = torch.from_numpy(replicas.rank_input(wl.x, rank)).pin_memory()
         dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
         x_dev = x_host.cuda()
         outs_host = [torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in dbb.outs]
@@ -211,11 +221,7 @@ def run_ours(args):
         barrier()
         wall = time.perf_counter() - t0
         clocks = sampler.stop() if sampler else None
-        ms = sum(a.elapsed_time(b) for a, b in ev)
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), device="cuda")
         launches = ctx.launch_count()
         h2d = x_host.numel() * 4 if e2e else 0
         d2h = sum(h.numel() * 4 for h in outs_host) if e2e else 0
@@ -223,7 +229,7 @@ def run_ours(args):
 
     def time_e2e(ratio, steps, warm):
         wl = workload(ratio)
-        x_host = torch.from_numpy(np.roll(wl.x, rank, axis=1).copy()).pin_memory()
+        x_host = torch.from_numpy(replicas.rank_input(wl.x, rank)).pin_memory()
         comp = torch.cuda.current_stream()
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
         sets = []
@@ -262,15 +268,12 @@ def run_ours(args):
         comp.wait_stream(s_out); comp.wait_stream(s_in)
         t_end.record(comp)
         barrier()
-        t = torch.tensor([t_begin.elapsed_time(t_end)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return dict(ms=float(t.item()), wl=wl, h2d=x_host.numel() * 4, d2h=sum(h.numel() * 4 for h in sets[0]["host"]))
+        return dict(ms=replicas.max_over_ranks(t_begin.elapsed_time(t_end), device="cuda"), wl=wl, h2d=x_host.numel() * 4, d2h=sum(h.numel() * 4 for h in sets[0]["host"]))
 
     sampler = ClockSampler(local) if rank == 0 else None
     main = time_ratio(args.ratio, K, Wm, sampler)
     ms_per_step = main["ms"] / K
-    value = world * wl_images(main["wl"]) * K / (main["ms"] / 1e3)
+    value = replicas.job_throughput(wl_images(main["wl"]), K, world, main["ms"])
 
     # per-kernel CUDA-event breakdown: a separate pass of the same K steps with events around every kernel
     ctx.profile_begin()
@@ -318,7 +321,7 @@ def run_ours(args):
     # the forward and copies the four stage maps device->host.  Two buffer sets and three streams let the copies of
     # neighbouring steps overlap the compute (PCIe is full duplex); the timed region is the whole pipeline of K steps.
     e2e = time_e2e(args.ratio, K, Wm)
-    e2e_value = world * wl_images(e2e["wl"]) * K / (e2e["ms"] / 1e3)
+    e2e_value = replicas.job_throughput(wl_images(e2e["wl"]), K, world, e2e["ms"])
 
     sweep = {}
     if args.sweep and world == 1:
@@ -343,12 +346,16 @@ def run_ours(args):
             dist.destroy_process_group()
         return
     line = {
-        "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "metric": METRIC if CONFIG == 3 else "two_branch_swin_backbone_images_per_sec_config%d" % CONFIG,
+        "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int8 MMA (int32 accumulate) + f32 epilogues", "data": "synthetic",
-        "config": {"workload": main["wl"].name, "model": "Swin-T two-branch backbone (96/192/384/768, 2/2/6/2)",
-                   "image": "800x1333", "tokens": [main["wl"].H, main["wl"].W], "batch_per_gpu": 1,
-                   "weights": "W4 (int8 container)", "act_bits_high_low": [8, 4], "low_ratio": args.ratio,
+        "config": {"workload": main["wl"].name,
+                   "model": "two-branch Swin backbone, dims %s depths %s" % (bbm.dims, bbm.depths),
+                   "tokens": [main["wl"].H, main["wl"].W], "batch_per_gpu": main["wl"].B,
+                   "weights": "W%d (int8 container)" % bbm.blocks[0].qkv.bits,
+                   "act_bits_high_low": [bbm.blocks[0].hi.bits, bbm.blocks[0].lo.bits], "low_ratio": args.ratio,
+                   "prune_ratio": (main["wl"].prune_ratios or [0.0])[0],
                    "l2": f"flushed between timed iterations ({L2_FLUSH_BYTES >> 20} MiB write)",
                    "parallelism": "replicas only (one image per GPU, no collective)"},
         "clocks": main["clocks"],
@@ -389,14 +396,23 @@ def oracle_sample(crop_h: int, crop_w: int, ratio: float):
 
 
 def cpu_baseline(full: bool, ratio: float = 0.5):
-    if full:
+    from oracle import oracle as orc
+    if full and CONFIG == 3:
         dt, imgs, thr, wl = oracle_sample(200, 334, ratio)
         sample = "one full forward of the same workload (1 image, 200x334 tokens)"
     else:
         dt, imgs, thr, wl = oracle_sample(50, 84, ratio)
-        sample = "one forward of a 50x84-token crop (6.3 % of the image's tokens), scaled by token count"
-    return {"value": round(imgs / dt, 5), "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample,
-            "seconds": round(dt, 3)}
+        sample = "one forward of a 50x84-token crop of the workload's images, scaled by token count"
+    out = {"value": round(imgs / dt, 5), "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample,
+           "seconds": round(dt, 3)}
+    # the same oracle on ONE thread, on the crop (the full image would take a minute)
+    n = orc.get_threads()
+    orc.set_threads(1)
+    dt1, imgs1, _, _ = oracle_sample(50, 84, ratio)
+    orc.set_threads(n)
+    out["single_thread"] = {"value": round(imgs1 / dt1, 5), "cores": 1, "seconds": round(dt1, 3),
+                            "sample": "50x84-token crop, scaled by token count"}
+    return out
 
 
 def run_reference(args):
@@ -404,23 +420,33 @@ def run_reference(args):
     if rank != 0:
         return
     K, Wm = args.steps, args.warmup
+    wl0 = workload(args.ratio)
+    H, W = wl0.H, wl0.W
+    # Every step is one oracle forward of a band of full-width rows of the workload's images (the whole image when the
+    # run fits a budget of about three minutes), scaled by token count.  Full-width bands keep enough windows per
+    # stage for the oracle's threads; a small square crop would leave most cores idle in the late stages.
+    dt_probe, _, thr, _ = oracle_sample(28, W, args.ratio)
+    est_full = dt_probe * H / 28.0
+    budget = 180.0
+    frac = min(1.0, budget / max(1e-9, (K + Wm) * est_full))
+    crop_h = H if frac >= 1.0 else max(28, int(H * frac / 28) * 28)
     for _ in range(Wm):
-        oracle_sample(50, 84, args.ratio)
+        oracle_sample(crop_h, W, args.ratio)
     t0 = time.perf_counter()
     imgs = 0.0
     for _ in range(K):
-        dt, im, thr, wl = oracle_sample(50, 84, args.ratio)
+        dt, im, thr, wl = oracle_sample(crop_h, W, args.ratio)
         imgs += im
     total = time.perf_counter() - t0
     value = imgs / total
+    sample = "each step = one oracle forward of %d of %d token rows (full width) of the workload, scaled by token count" % (crop_h, H)
     line = {
-        "impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "impl": "reference", "metric": METRIC if CONFIG == 3 else "two_branch_swin_backbone_images_per_sec_config%d" % CONFIG,
+        "value": round(value, 5), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": K, "warmup": Wm, "ms_per_step": round(1e3 * total / K, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int32/int64 integer + f32", "data": "synthetic",
-        "config": {"workload": wl.name, "low_ratio": args.ratio,
-                   "sample": "each step = one oracle forward of a 50x84-token crop (6.3 % of the tokens), scaled by token count"},
-        "cpu_baseline": {"value": round(value, 5), "unit": UNIT, "cores": thr, "kind": "oracle",
-                         "sample": "50x84-token crop per step, scaled by token count"},
+        "config": {"workload": wl.name, "low_ratio": args.ratio, "sample": sample},
+        "cpu_baseline": {"value": round(value, 5), "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 5), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -433,9 +459,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ratio", type=float, default=0.5)
+    ap.add_argument("--config", type=int, default=3, choices=[3, 4, 5],
+                    help="3: Swin-T 800x1333 B=1 (the metric's workload); 4: Swin-S 1024^2 B=4 A4/A2 + 20 %% pruned; 5: Swin-B 1536^2 B=2")
     ap.add_argument("--no-sweep", dest="sweep", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     args = ap.parse_args()
+    global CONFIG
+    CONFIG = args.config
+    if CONFIG != 3:
+        args.sweep = False
     if args.impl == "reference":
         run_reference(args)
     else:
