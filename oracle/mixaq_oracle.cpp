@@ -529,6 +529,37 @@ void orc_merge_forward(const orc_merge* m, const float* x, int B, int H, int W, 
   }
 }
 
+// patch embedding: 4x4 patches (zero padding to multiples of 4) -> quantize -> integer projection -> + bias -> LN
+void orc_patch_embed(const orc_embed* e, const float* img, int B, int Hi, int Wi, float* x0) {
+  const int H = (Hi + 3) / 4, W = (Wi + 3) / 4, K = 48, N = e->proj.out_f;
+#pragma omp parallel for schedule(static)
+  for (long tok = 0; tok < (long)B * H * W; ++tok) {
+    const int b = (int)(tok / ((long)H * W)), r = (int)(tok % ((long)H * W));
+    const int ty = r / W, tx = r % W;
+    std::vector<float> v(K, 0.0f), t(N), y(N);
+    for (int ky = 0; ky < 4; ++ky)
+      for (int kx = 0; kx < 4; ++kx) {
+        const int yy = 4 * ty + ky, xx = 4 * tx + kx;
+        if (yy < Hi && xx < Wi)
+          for (int c = 0; c < 3; ++c) v[(ky * 4 + kx) * 3 + c] = img[(((long)b * Hi + yy) * Wi + xx) * 3 + c];
+      }
+    if (e->quant) {
+      std::vector<uint8_t> a(K);
+      orc_quantize(v.data(), K, e->in, a.data());
+      std::vector<int32_t> acc(N);
+      int_linear(a.data(), 1, K, e->in.zp, e->proj, acc.data());
+      for (int n = 0; n < N; ++n) {
+        const float d = (float)acc[n] * (e->in.scale * e->proj.scale[n]);
+        t[n] = d + e->bias[n];
+      }
+    } else {
+      fp_linear(v.data(), 1, K, e->proj, e->bias, t.data());
+    }
+    layernorm_row(t.data(), N, e->ln_g, e->ln_b, y.data());
+    std::memcpy(x0 + tok * N, y.data(), N * sizeof(float));
+  }
+}
+
 void orc_backbone_forward(int num_stages, const int* depths, const orc_block* blocks, const orc_merge* merges,
                           const float* x0, float* const* stage_out, int B, int H0, int W0,
                           const double* low_ratio_per_pair, const double* prune_ratio_per_pair) {

@@ -67,6 +67,14 @@ typedef struct {
 
 typedef struct { const float *ln_g, *ln_b; orc_aq in; orc_linear red; int quant; } orc_merge;
 
+/* Patch embedding in front of the backbone (the stem of the Swin backbone the paper quantizes; its cost belongs to the
+ * layers the method does not reduce, Appendix 6.2): 4x4 non-overlapping patches of an [B][Hi][Wi][3] image (zero
+ * padded to multiples of 4), patch vector index (ky*4 + kx)*3 + c, quantized with `in`, integer projection
+ * [C0][48], then t = (float)acc * (s_in*s_w[n]) + bias[n] (two rounded operations), then LayerNorm(C0).
+ * quant = 0: the same in floating point (binary64 accumulation).  Paper silent on all numerics: parity unpinned by
+ * the paper, pinned to numpy convolution + LayerNorm in tests. */
+typedef struct { const float *ln_g, *ln_b, *bias; orc_aq in; orc_linear proj; int quant; } orc_embed;
+
 /* ---- primitives (each pinned separately) ---- */
 int   orc_low_count(double ratio, int n);
 void  orc_quantize(const float* x, long n, orc_aq q, uint8_t* codes);
@@ -105,6 +113,7 @@ void  orc_merge_forward(const orc_merge* m, const float* x, int B, int H, int W,
 void  orc_backbone_forward(int num_stages, const int* depths, const orc_block* blocks, const orc_merge* merges,
                            const float* x0, float* const* stage_out, int B, int H0, int W0,
                            const double* low_ratio_per_pair, const double* prune_ratio_per_pair);
+void  orc_patch_embed(const orc_embed* e, const float* img, int B, int Hi, int Wi, float* x0 /* [B][ceil(Hi/4)][ceil(Wi/4)][C0] */);
 void  orc_set_threads(int n);
 int   orc_get_threads(void);
 #ifdef __cplusplus

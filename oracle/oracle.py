@@ -63,6 +63,11 @@ class MergeS(C.Structure):
     _fields_ = [("ln_g", C.c_void_p), ("ln_b", C.c_void_p), ("in_", AQ), ("red", LinearS), ("quant", C.c_int)]
 
 
+class EmbedS(C.Structure):
+    _fields_ = [("ln_g", C.c_void_p), ("ln_b", C.c_void_p), ("bias", C.c_void_p), ("in_", AQ), ("proj", LinearS),
+                ("quant", C.c_int)]
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -335,6 +340,19 @@ def backbone_forward(bb, x, low_ratios, prune_ratios=None, quant=True):
         pr = (C.c_double * npairs)(*([float(r) for r in prune_ratios] + [0.0] * (npairs - len(prune_ratios))))
     lib().orc_backbone_forward(ns, depths, blocks, merges, _p(x), ptrs, B, H, W, lr, pr)
     return outs
+
+
+def patch_embed(e, img, quant=True):
+    """e: object with ln_g, ln_b, bias, aq, proj (codes [C0][48], scale).  img: [B][Hi][Wi][3] float32."""
+    img = np.ascontiguousarray(img, np.float32)
+    B, Hi, Wi, ch = img.shape
+    assert ch == 3
+    keep = _Keep()
+    es = EmbedS(keep.arr(e.ln_g, np.float32), keep.arr(e.ln_b, np.float32), keep.arr(e.bias, np.float32), _aq(e.aq),
+                _linear(keep, e.proj), 1 if quant else 0)
+    out = np.empty((B, (Hi + 3) // 4, (Wi + 3) // 4, e.proj.codes.shape[0]), np.float32)
+    lib().orc_patch_embed(C.byref(es), _p(img), B, Hi, Wi, _p(out))
+    return out
 
 
 def set_threads(n):

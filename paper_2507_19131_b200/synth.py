@@ -95,6 +95,31 @@ class Merge:
 
 
 @dataclass
+class Embed:
+    ln_g: np.ndarray
+    ln_b: np.ndarray
+    bias: np.ndarray
+    aq: AQ
+    proj: Linear                # [C0, 48]: 4x4 patch of 3 channels, index (ky*4 + kx)*3 + c
+
+
+def make_embed(rng, c0: int, w_bits: int = 8, bits: int = 8, pixel_range: float = 3.0) -> Embed:
+    """Stem parameters: N(0, 0.02^2) projection quantized per output channel, LN gamma/beta as elsewhere, and an input
+    quantizer for standardised pixels (ImageNet-style mean/std normalisation puts them in about +-3)."""
+    return Embed(_vec(rng, c0, 1.0, 0.02), _vec(rng, c0, 0.0, 0.02), _vec(rng, c0, 0.0, 0.02),
+                 make_aq(-pixel_range, pixel_range, bits), make_linear(rng, c0, 48, w_bits))
+
+
+def input_image(seed: int, B, Hi, Wi) -> np.ndarray:
+    """A standardised synthetic image [B][Hi][Wi][3]: smooth blobs plus pixel noise."""
+    rng = np.random.default_rng(seed)
+    img = rng.standard_normal((B, Hi, Wi, 3), dtype=F32) * F32(0.5)
+    for b in range(B):
+        img[b] += (2.0 * blob_map(rng, Hi, Wi) - 0.5).astype(F32)[..., None]
+    return img
+
+
+@dataclass
 class Backbone:
     dims: List[int]
     depths: List[int]

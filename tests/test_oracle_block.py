@@ -320,3 +320,59 @@ def test_backbone_shares_the_stage_entry_energy_across_the_stage(orc):
             cur = orc.block_forward(bb.blocks[k], cur, wl.low_ratios[k // 2], wl.prune_ratios[k // 2], energy_map=e).y
             k += 1
         assert np.array_equal(outs[s], cur)
+
+
+# ------------------------------------------------------------------------------------------------
+# patch embedding (the stem in front of the backbone) and output norms
+# ------------------------------------------------------------------------------------------------
+def _embed_numpy_fp(e, img):
+    """4x4 stride-4 convolution written as a reshape + matmul in binary64, then LayerNorm in binary64."""
+    B, Hi, Wi, _ = img.shape
+    Hp, Wp = -(-Hi // 4) * 4, -(-Wi // 4) * 4
+    pad = np.zeros((B, Hp, Wp, 3), np.float64)
+    pad[:, :Hi, :Wi] = img
+    patches = pad.reshape(B, Hp // 4, 4, Wp // 4, 4, 3).transpose(0, 1, 3, 2, 4, 5).reshape(B, Hp // 4, Wp // 4, 48)
+    w = e.proj.codes.astype(np.float64) * e.proj.scale.astype(np.float64)[:, None]
+    t = patches @ w.T + e.bias.astype(np.float64)
+    mu = t.mean(-1, keepdims=True)
+    var = ((t - mu) ** 2).mean(-1, keepdims=True)
+    return (t - mu) / np.sqrt(var + 1e-5) * e.ln_g + e.ln_b
+
+
+@pytest.mark.parametrize("Hi,Wi", [(16, 20), (13, 18), (7, 5)])
+def test_patch_embed_fp_mode_is_a_strided_convolution_plus_layernorm(orc, Hi, Wi):
+    e = synth.make_embed(np.random.default_rng(3), 32)
+    img = synth.input_image(4, 2, Hi, Wi)
+    got = orc.patch_embed(e, img, quant=False)
+    want = _embed_numpy_fp(e, img)
+    assert got.shape == want.shape == (2, -(-Hi // 4), -(-Wi // 4), 32)
+    assert np.abs(got - want).max() < 2e-5
+
+
+def test_patch_embed_quantized_from_pinned_primitives_and_onehot(orc):
+    e = synth.make_embed(np.random.default_rng(5), 32)
+    img = synth.input_image(6, 1, 12, 9)                          # 9 -> padded to 12 columns
+    got = orc.patch_embed(e, img, quant=True)
+    pad = np.zeros((1, 12, 12, 3), F32)
+    pad[:, :, :9] = img
+    patches = pad.reshape(1, 3, 4, 3, 4, 3).transpose(0, 1, 3, 2, 4, 5).reshape(-1, 48)
+    codes = orc.quantize(patches, e.aq)
+    acc = orc.int_gemm(codes, e.aq.zp, e.proj.codes)
+    t = (acc.astype(F32) * (F32(e.aq.scale) * e.proj.scale)[None, :]).astype(F32) + e.bias[None, :]
+    want = orc.layernorm(t.astype(F32), e.ln_g, e.ln_b).reshape(got.shape)
+    assert np.array_equal(got, want)
+    # close to the floating-point stem at 8 bits
+    assert np.abs(got - orc.patch_embed(e, img, quant=False)).max() < 0.15
+    # one-hot projection rows: output channel n sees exactly pixel k_n of the patch (dequantized), before the norm
+    e2 = synth.make_embed(np.random.default_rng(7), 32)
+    e2.proj.codes[:] = 0
+    for n in range(32):
+        e2.proj.codes[n, n] = 1
+    e2.proj.scale[:] = 1.0
+    e2.bias[:] = 0.0
+    e2.ln_g[:] = 1.0
+    e2.ln_b[:] = 0.0
+    g2 = orc.patch_embed(e2, img, quant=True).reshape(-1, 32)
+    deq = orc.dequantize(codes[:, :32], e2.aq)
+    want2 = orc.layernorm(deq, e2.ln_g, e2.ln_b)
+    assert np.array_equal(g2, want2)
