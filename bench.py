@@ -340,6 +340,33 @@ def run_ours(args):
                      "equivalent_act_bits": round(cm.equivalent_act_bits([r] * len(pair_g), 8.0, pair_g, fixed_g), 3)}
             for r in (SWEEP if args.sweep else [args.ratio])}
 
+    # the steps on either side of the path (patch embedding of the raw image, LayerNorm of the four stage maps)
+    stem = None
+    if CONFIG == 3 and world == 1:
+        from paper_2507_19131_b200 import synth
+        rng = np.random.default_rng(77)
+        emb = synth.make_embed(rng, bbm.dims[0])
+        de = mq.DeviceEmbed(ctx, emb)
+        img = torch.from_numpy(synth.input_image(78, main["wl"].B, 800, 1333)).cuda()
+        gb = [(torch.ones(c, device="cuda"), torch.zeros(c, device="cuda")) for c in bbm.dims]
+        outs = main["dbb"].outs
+        x0 = mq.embed_forward(ctx, de, img)
+
+        def timed(fn, n=20):
+            for _ in range(3):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(n):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) * 1e3 / n
+        stem = {"patch_embed_us": round(timed(lambda: mq.embed_forward(ctx, de, img, x0)), 2),
+                "stage_norms_us": round(timed(lambda: [mq.norm_forward(ctx, g, b, o, o) for (g, b), o in zip(gb, outs)]), 2),
+                "note": "800x1333x3 image -> 200x334x96 tokens (3 launches); LayerNorm of the 4 stage maps (4 launches); "
+                        "stream launches, not part of `value`"}
+
     status = ctx.device_status()
     if rank != 0:
         if world > 1:
@@ -367,6 +394,7 @@ def run_ours(args):
         "kernels": kernels,
         "low_ratio_sweep_images_per_sec": sweep,
         "paper_cost_model": cost,
+        "stem_and_norms": stem,
         "device_status": status,
     }
     if args.cpu_baseline and world == 1:

@@ -75,6 +75,12 @@ typedef struct {
  * Appendix 6.2: their cost is not reduced by the method.) */
 typedef struct { const float *ln_g, *ln_b; mixaq_aq in; mixaq_linear reduction; void* prepared; } mixaq_merge_params;
 
+/* Patch embedding in front of the backbone: 4x4 patches of an [B][Hi][Wi][3] binary32 image (zero padded to
+ * multiples of 4; patch vector index (ky*4 + kx)*3 + c) -> quantize (`in`, all tokens at the high bit width) ->
+ * integer projection [C0][48] -> (float)acc * (s_in*s_w[n]) + bias[n] -> LayerNorm(C0).  Like patch merging it is one
+ * of the layers whose cost the method does not reduce (Appendix 6.2).  C0 must be a multiple of 32. */
+typedef struct { const float *ln_g, *ln_b, *bias; mixaq_aq in; mixaq_linear proj; void* prepared; } mixaq_embed_params;
+
 typedef struct {
   const int32_t* energy;   /* optional [B][H][W] token energies computed at stage entry (Section 3.2: the score is
                               computed once per stage and shared); NULL: score this block's own input x      */
@@ -168,6 +174,17 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
 #define MIXAQ_STATIC_SCRATCH_BYTES (8u << 20)
 mixaq_status mixaq_merge_forward_static(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
                                         int B, int H, int W, void* cuda_stream);
+
+/* ---- patch embedding (the step in front of the path) and LayerNorm of a stage output (the step behind it).
+ *      image [B][Hi][Wi][3] -> x0 [B][ceil(Hi/4)][ceil(Wi/4)][C0], the input of mixaq_backbone_forward.
+ *      mixaq_norm_forward: y = LayerNorm(x) over the last axis of a [rows][C] binary32 matrix (x and y may alias). ---- */
+size_t       mixaq_embed_prepared_bytes(const mixaq_embed_params* p);
+mixaq_status mixaq_embed_prepare(mixaq_ctx* ctx, const mixaq_embed_params* p, void* cuda_stream);
+size_t       mixaq_embed_workspace_bytes(const mixaq_embed_params* p, int B, int Hi, int Wi);
+mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, const float* image, float* x0,
+                                 int B, int Hi, int Wi, void* workspace, size_t workspace_bytes, void* cuda_stream);
+mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float* beta, const float* x, float* y,
+                                long rows, int C, void* cuda_stream);
 
 /* ---- the backbone: for every stage [merge] -> stage energy -> blocks; one ratio per pair of consecutive
  *      blocks (Section 3.3), optional prune ratio per pair (Section 3.4).  x0 is the [B][H0][W0][C0] map after the

@@ -22,6 +22,8 @@ EXPORTS = [
     "mixaq_merge_workspace_bytes", "mixaq_merge_forward", "mixaq_backbone_workspace_bytes",
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
+    "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
+    "mixaq_norm_forward",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -60,6 +62,11 @@ class MergeS(C.Structure):
                 ("prepared", C.c_void_p)]
 
 
+class EmbedS(C.Structure):
+    _fields_ = [("ln_g", C.c_void_p), ("ln_b", C.c_void_p), ("bias", C.c_void_p), ("in_", AQ), ("proj", LinearS),
+                ("prepared", C.c_void_p)]
+
+
 class SelectOpts(C.Structure):
     _fields_ = [("energy", C.c_void_p), ("reverse", C.c_int)]
 
@@ -94,7 +101,8 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.mixaq_last_error.restype = C.c_char_p
         L.mixaq_profile_category_name.restype = C.c_char_p
-        for n in ("mixaq_block_prepared_bytes", "mixaq_merge_prepared_bytes", "mixaq_block_workspace_bytes",
+        for n in ("mixaq_embed_prepared_bytes", "mixaq_embed_workspace_bytes",
+                  "mixaq_block_prepared_bytes", "mixaq_merge_prepared_bytes", "mixaq_block_workspace_bytes",
                   "mixaq_merge_workspace_bytes", "mixaq_backbone_workspace_bytes"):
             getattr(L, n).restype = C.c_size_t
         L.mixaq_low_count.argtypes = [C.c_float, C.c_int]
@@ -314,6 +322,46 @@ def merge_forward(ctx: Context, dm: DeviceMerge, x: torch.Tensor) -> torch.Tenso
     ws = torch.empty(need, dtype=torch.uint8, device=x.device)
     ctx.check(lib().mixaq_merge_forward(ctx.h, C.byref(dm.s), _ptr(x), _ptr(y), B, H, W, _ptr(ws), C.c_size_t(need),
                                         _stream_ptr()), "merge_forward")
+    return y
+
+
+class DeviceEmbed:
+    """Stem parameters on the device, prepared (mixaq_embed_prepare)."""
+
+    def __init__(self, ctx: Context, e):
+        self.ctx, self.e = ctx, e
+        self.dev = _Dev(ctx.device)
+        self.s = EmbedS(self.dev.up(e.ln_g, np.float32), self.dev.up(e.ln_b, np.float32), self.dev.up(e.bias, np.float32),
+                        _aq(e.aq), _linear(self.dev, e.proj), None)
+        self.s.prepared = self.dev.empty(lib().mixaq_embed_prepared_bytes(C.byref(self.s)))
+        ctx.check(lib().mixaq_embed_prepare(ctx.h, C.byref(self.s), _stream_ptr()), "embed_prepare")
+        self._ws = None
+
+
+def embed_forward(ctx: Context, de: DeviceEmbed, image: torch.Tensor, x0: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """mixaq_embed_forward: image [B,Hi,Wi,3] float32 -> x0 [B,ceil(Hi/4),ceil(Wi/4),C0]."""
+    assert image.is_cuda and image.dtype == torch.float32 and image.is_contiguous() and image.shape[-1] == 3
+    B, Hi, Wi, _ = image.shape
+    c0 = de.e.proj.codes.shape[0]
+    if x0 is None:
+        x0 = torch.empty((B, (Hi + 3) // 4, (Wi + 3) // 4, c0), dtype=torch.float32, device=image.device)
+    need = lib().mixaq_embed_workspace_bytes(C.byref(de.s), B, Hi, Wi)
+    if de._ws is None or de._ws.numel() < need:
+        de._ws = torch.empty(need, dtype=torch.uint8, device=image.device)
+    ctx.check(lib().mixaq_embed_forward(ctx.h, C.byref(de.s), _ptr(image), _ptr(x0), B, Hi, Wi, _ptr(de._ws),
+                                        C.c_size_t(de._ws.numel()), _stream_ptr()), "embed_forward")
+    return x0
+
+
+def norm_forward(ctx: Context, gamma: torch.Tensor, beta: torch.Tensor, x: torch.Tensor,
+                 y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """mixaq_norm_forward: LayerNorm over the last axis of a float32 tensor (a stage's output map)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    if y is None:
+        y = torch.empty_like(x)
+    Cc = x.shape[-1]
+    ctx.check(lib().mixaq_norm_forward(ctx.h, _ptr(gamma), _ptr(beta), _ptr(x), _ptr(y), C.c_long(x.numel() // Cc), Cc,
+                                       _stream_ptr()), "norm_forward")
     return y
 
 

@@ -43,6 +43,14 @@ struct MergeGatherArgs {
 void launch_merge_gather(const MergeGatherArgs& a, cudaStream_t st);
 void launch_copy_rows(const float* x, float* y, const int32_t* rowsrc, int M, int C, cudaStream_t st);
 
+// ---- stem and output norms ---------------------------------------------------------------------------
+struct PatchGatherArgs { const float* img; uint8_t* out; AQ q; int B, Hi, Wi; };   // out: [tokens][64] codes
+void launch_patch_gather(const PatchGatherArgs& a, cudaStream_t st);
+// y = LayerNorm(x + bias), binary32 in and out, rows x C; bias nullable.  false: C not supported.
+bool launch_bias_ln(const float* x, const float* bias, const float* gamma, const float* beta, float* y, long rows,
+                    int C, cudaStream_t st);
+void launch_pad_weights(const int8_t* w, int N, int K, int Kp, int8_t* out, cudaStream_t st);
+
 // ---- integer GEMM with fused epilogues ----------------------------------------------------------
 enum EpiMode { EPI_QKV = 0, EPI_PROJ = 1, EPI_FC1 = 2, EPI_FC2 = 3, EPI_MERGE = 4 };
 

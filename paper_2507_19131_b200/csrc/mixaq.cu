@@ -679,6 +679,87 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   return check_cuda(ctx, "backbone_forward");
 }
 
+// -------------------------------------------------------------------------------------------------
+// stem and output norms
+namespace {
+constexpr int EMBED_K = 48, EMBED_KP = 64;     // patch vector, padded to a multiple of 32 codes
+struct EmbedPrepared { int8_t* w; float* mult; int32_t* zc; size_t bytes; };
+EmbedPrepared carve_embed(const mixaq_embed_params* p, void* base) {
+  EmbedPrepared r; Carver c(base);
+  const int N = p->proj.out_features;
+  r.w = c.take<int8_t>((size_t)N * EMBED_KP); r.mult = c.take<float>(N); r.zc = c.take<int32_t>(N);
+  r.bytes = c.off;
+  return r;
+}
+bool embed_ok(const mixaq_embed_params* p) {
+  return p && p->ln_g && p->ln_b && p->bias && p->proj.codes && p->proj.scale && p->proj.in_features == EMBED_K &&
+         p->proj.out_features > 0 && p->proj.out_features % 32 == 0 && ln_dim_supported(p->proj.out_features) &&
+         bits_ok(p->in.bits) && aq_ok(p->in, p->in.bits) && p->in.bits == 8;
+}
+}  // namespace
+
+size_t mixaq_embed_prepared_bytes(const mixaq_embed_params* p) {
+  if (!p || p->proj.out_features <= 0) return 0;
+  return carve_embed(p, nullptr).bytes;
+}
+
+mixaq_status mixaq_embed_prepare(mixaq_ctx* ctx, const mixaq_embed_params* p, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  if (!embed_ok(p) || !p->prepared) return fail(ctx, MIXAQ_INVALID_ARG, "embed params incomplete (8-bit input, [C0][48] projection, C0 % 32 == 0)");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  EmbedPrepared pr = carve_embed(p, p->prepared);
+  const int N = p->proj.out_features;
+  launch_pad_weights(p->proj.codes, N, EMBED_K, EMBED_KP, pr.w, st);
+  launch_prepare_linear(pr.w, p->proj.scale, N, EMBED_KP, p->in.scale, p->in.zero_point, pr.mult, pr.zc, st);
+  return check_cuda(ctx, "embed_prepare");
+}
+
+size_t mixaq_embed_workspace_bytes(const mixaq_embed_params* p, int B, int Hi, int Wi) {
+  if (!p || B <= 0 || Hi <= 0 || Wi <= 0 || p->proj.out_features <= 0) return 0;
+  const size_t toks = (size_t)B * ((Hi + 3) / 4) * ((Wi + 3) / 4);
+  return align_up(toks * EMBED_KP) + align_up(toks * p->proj.out_features * sizeof(float));
+}
+
+mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, const float* image, float* x0,
+                                 int B, int Hi, int Wi, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  if (!embed_ok(p) || !p->prepared) return fail(ctx, MIXAQ_INVALID_ARG, "embed params incomplete");
+  if (!image || !x0 || !workspace || B <= 0 || Hi <= 0 || Wi <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "embed: bad argument");
+  if (mixaq_embed_workspace_bytes(p, B, Hi, Wi) > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "embed workspace");
+  const size_t toks = (size_t)B * ((Hi + 3) / 4) * ((Wi + 3) / 4);
+  if (toks >= (size_t)1 << 31) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many tokens");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int N = p->proj.out_features;
+  Carver c(workspace);
+  uint8_t* codes = c.take<uint8_t>(toks * EMBED_KP);
+  float* t = c.take<float>(toks * N);
+  EmbedPrepared pr = carve_embed(p, p->prepared);
+  g_launches = 0;
+  PatchGatherArgs pg; pg.img = image; pg.out = codes; pg.q = to_aq(p->in); pg.B = B; pg.Hi = Hi; pg.Wi = Wi;
+  launch_patch_gather(pg, st);
+  GemmArgs ga;
+  ga.status = ctx->d_status;
+  ga.w = pr.w; ga.N = N; ga.K = EMBED_KP; ga.C = N; ga.mode = EPI_MERGE;      // dequantize only: acc * mult
+  fill_gemm_branch(ga.br[0], codes, (int)toks, 8, pr.mult, pr.zc, nullptr);
+  ga.br[0].out_f = t;
+  fill_gemm_branch(ga.br[1], nullptr, 0, 8, pr.mult, pr.zc, nullptr);
+  if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)");
+  if (!launch_bias_ln(t, p->bias, p->ln_g, p->ln_b, x0, (long)toks, N, st)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "embed: unsupported C0");
+  ctx->launches = g_launches;
+  return check_cuda(ctx, "embed_forward");
+}
+
+mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float* beta, const float* x, float* y,
+                                long rows, int C, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  if (!gamma || !beta || !x || !y || rows <= 0 || C <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "norm: bad argument");
+  g_launches = 0;
+  if (!launch_bias_ln(x, nullptr, gamma, beta, y, rows, C, (cudaStream_t)cuda_stream))
+    return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "norm: unsupported C");
+  ctx->launches = g_launches;
+  return check_cuda(ctx, "norm_forward");
+}
+
 mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   ctx->graph_cache = enabled != 0;

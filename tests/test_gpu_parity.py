@@ -215,6 +215,50 @@ def test_config5_swin_b_1536_full_size(orc, mq, ctx):
     _full_backbone_case(orc, mq, ctx, synth.config5(ratio=0.5))
 
 
+@pytest.mark.parametrize("B,Hi,Wi,C0", [(2, 16, 20, 32), (1, 13, 18, 96), (1, 7, 5, 32), (1, 800, 1333, 96)])
+def test_patch_embed_parity(orc, mq, ctx, B, Hi, Wi, C0):
+    """The stem in front of the backbone (image -> x0), including sizes that need zero padding and the full
+    800 x 1333 image of the benchmark workload."""
+    e = synth.make_embed(np.random.default_rng(C0 + Hi), C0)
+    img = synth.input_image(Hi + Wi, B, Hi, Wi)
+    de = mq.DeviceEmbed(ctx, e)
+    got = mq.embed_forward(ctx, de, dev(img)).cpu().numpy()
+    want = orc.patch_embed(e, img)
+    assert got.shape == want.shape
+    assert_close_rel(got, want)
+    assert np.array_equal(got, want)
+
+
+def test_stage_output_norm_parity(orc, mq, ctx):
+    rng = np.random.default_rng(9)
+    for (rows_shape, Cc) in [((2, 9, 11), 96), ((1, 25, 42), 768), ((3, 5, 7), 192)]:
+        x = (rng.standard_normal(rows_shape + (Cc,), dtype=F32) * F32(3.0) + F32(0.5)).astype(F32)
+        g = (1.0 + 0.1 * rng.standard_normal(Cc)).astype(F32)
+        b = (0.1 * rng.standard_normal(Cc)).astype(F32)
+        got = mq.norm_forward(ctx, dev(g), dev(b), dev(x)).cpu().numpy()
+        want = orc.layernorm(x, g, b)
+        assert np.array_equal(got, want)
+
+
+def test_image_to_normed_stage_maps_end_to_end(orc, mq, ctx):
+    """image -> stem -> two-branch backbone -> per-stage output norms, against the same chain of oracle calls."""
+    wl = synth.tiny_backbone(ratio=0.4, prune=0.2)
+    rng = np.random.default_rng(11)
+    e = synth.make_embed(rng, wl.backbone.dims[0])
+    img = synth.input_image(12, wl.B, 4 * wl.H - 1, 4 * wl.W - 2)          # pads up to (4H, 4W)
+    norms = [((1.0 + 0.05 * rng.standard_normal(c)).astype(F32), (0.05 * rng.standard_normal(c)).astype(F32)) for c in wl.backbone.dims]
+    x0_ref = orc.patch_embed(e, img)
+    want = [orc.layernorm(o, g, b) for o, (g, b) in zip(orc.backbone_forward(wl.backbone, x0_ref, wl.low_ratios, wl.prune_ratios), norms)]
+    de = mq.DeviceEmbed(ctx, e)
+    x0 = mq.embed_forward(ctx, de, dev(img))
+    assert tuple(x0.shape) == (wl.B, wl.H, wl.W, wl.backbone.dims[0])
+    dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+    outs = mq.backbone_forward(ctx, dbb, x0, wl.low_ratios, wl.prune_ratios)
+    got = [mq.norm_forward(ctx, dev(g), dev(b), o).cpu().numpy() for o, (g, b) in zip(outs, norms)]
+    for gg, ww in zip(got, want):
+        assert np.array_equal(gg, ww)
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
     import ctypes as C
     blk = synth.make_block(np.random.default_rng(40), 32, 1, 0, 8, 8, 4)
