@@ -53,6 +53,99 @@ __global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo, int 
   }
 }
 
+// The same LayerNorm for large batches of narrow rows: G lanes share a row and a warp works on 32/G rows at once.
+// Lane j of a row's group owns the partial sums of indices P*j .. P*j+P-1 (P = 32/G) of the 32 interleaved
+// partials, i.e. of every 32-channel group the P contiguous channels 32i + P*j ..: vector loads, whole bytes of
+// codes per lane, and the butterfly (offsets 16, 8, 4, 2, 1 on the partial index) becomes log2(G) exchanges
+// between lanes followed by a tree inside the lane -- the same additions in the same order.
+template <int NG, int G>
+__global__ void __launch_bounds__(256, 4) k_ln_quant_g(LnBranch hi, LnBranch lo, int blocks_hi) {
+  constexpr int C = NG * 32, P = 32 / G, ROWS = 32 / G;     // channels, partials per lane, rows per warp
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int j = lane % G, rw = lane / G;
+  const bool is_hi = (int)blockIdx.x < blocks_hi;
+  const LnBranch& br = is_hi ? hi : lo;
+  const int M = br.M;
+  const int blk = is_hi ? blockIdx.x : blockIdx.x - blocks_hi;
+  const int m0 = (blk * 8 + warp) * ROWS;
+  if (m0 >= M) return;
+  const int m = m0 + rw;
+  const AQ q = br.q;
+  const int bits = q.bits;
+  long srow = -1;
+  if (m < M) srow = br.rowsrc ? (long)br.rowsrc[m] : (long)m;
+  float x[NG][P];
+  const float* row = br.src + (srow < 0 ? 0 : srow) * C + P * j;
+#pragma unroll
+  for (int i = 0; i < NG; ++i) {
+#pragma unroll
+    for (int v4 = 0; v4 < P / 4; ++v4) {
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (srow >= 0) a = __ldg(reinterpret_cast<const float4*>(row + 32 * i) + v4);
+      x[i][4 * v4] = a.x; x[i][4 * v4 + 1] = a.y; x[i][4 * v4 + 2] = a.z; x[i][4 * v4 + 3] = a.w;
+    }
+  }
+  // partial sums in channel order, then the butterfly: lanes first (offsets 16 .. P), then inside the lane
+  auto reduce32 = [&](float (&p)[P]) -> float {
+#pragma unroll
+    for (int o = G / 2; o >= 1; o >>= 1)
+#pragma unroll
+      for (int k = 0; k < P; ++k) p[k] = __fadd_rn(p[k], __shfl_xor_sync(0xffffffffu, p[k], o));
+#pragma unroll
+    for (int o = P / 2; o >= 1; o >>= 1)
+#pragma unroll
+      for (int k = 0; k < o; ++k) p[k] = __fadd_rn(p[k], p[k + o]);
+    return p[0];
+  };
+  float p[P];
+#pragma unroll
+  for (int k = 0; k < P; ++k) {
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NG; ++i) s = __fadd_rn(s, x[i][k]);
+    p[k] = s;
+  }
+  const float mean = __fdiv_rn(reduce32(p), (float)C);
+#pragma unroll
+  for (int k = 0; k < P; ++k) {
+    float v = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NG; ++i) { const float d = __fsub_rn(x[i][k], mean); v = __fmaf_rn(d, d, v); }
+    p[k] = v;
+  }
+  const float var = __fdiv_rn(reduce32(p), (float)C);
+  const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, 1e-5f)));
+  if (m >= M) return;
+  uint8_t* out = br.out + (long)m * (C * bits / 8) + (P * j) * bits / 8;
+  const uint32_t kpack = pack_const(q.zp, bits);
+  const uint32_t zpat = quant_magic(0.0f, q);      // pad token: zero after the normalisation
+  const int per = 32 / bits;                       // codes per 32-bit word
+#pragma unroll
+  for (int i = 0; i < NG; ++i) {
+    uint32_t w0 = kpack, w1 = kpack;
+#pragma unroll
+    for (int v4 = 0; v4 < P / 4; ++v4) {
+      const float4 g4 = __ldg(reinterpret_cast<const float4*>(br.gamma + 32 * i + P * j) + v4);
+      const float4 b4 = __ldg(reinterpret_cast<const float4*>(br.beta + 32 * i + P * j) + v4);
+      const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int k = 4 * v4 + e;
+        const uint32_t pat = srow < 0 ? zpat : quant_magic(ln_apply(x[i][k], mean, rstd, gg[e], bb[e]), q);
+        if (k < per) w0 += pat << (bits * k);
+        else         w1 += pat << (bits * (k - per));
+      }
+    }
+    // P codes of `bits` bits: P*bits/8 whole bytes (the launcher only picks G with P*bits >= 8)
+    uint8_t* dst = out + 32 * i * bits / 8;
+    const int nbytes = P * bits / 8;
+    if (nbytes == 8) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
+    else if (nbytes == 4) *reinterpret_cast<uint32_t*>(dst) = w0;
+    else if (nbytes == 2) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)w0;
+    else *dst = (uint8_t)w0;
+  }
+}
+
 // patch merging: token (b, y2, x2) of the output gathers (2y2+dy, 2x2+dx) for (dy,dx) = (0,0),(1,0),(0,1),(1,1)
 // in this order along the channel axis; neighbours outside the map are zeros (they do take part in the LN).
 template <int NPL>   // NPL = 4C/32
@@ -115,8 +208,30 @@ void launch_ln_npl(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
 #define MIXAQ_NPL_CASE(n, KERNEL, ...) case n: KERNEL<n><<<grid, 256, 0, st>>>(__VA_ARGS__); break;
 #define MIXAQ_LN_CASE(n, rmax) case n: launch_ln_npl<n, rmax>(hi, lo, st); break;
 
+template <int NG, int G>
+void launch_ln_g(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
+  const int rpb = 8 * (32 / G);                              // rows per block: 8 warps x 32/G rows
+  const int bh = (hi.M + rpb - 1) / rpb, bl = (lo.M + rpb - 1) / rpb;
+  k_ln_quant_g<NG, G><<<bh + bl, 256, 0, st>>>(hi, lo, bh);
+}
+
 void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st) {
   if (hi.M + lo.M == 0) return;
+  // narrow rows in large batches: several lanes per row, provided every lane then stores whole bytes of codes
+  const int rows = hi.M + lo.M;
+  const int min_bits = hi.M > 0 && lo.M > 0 ? (hi.q.bits < lo.q.bits ? hi.q.bits : lo.q.bits) : (hi.M > 0 ? hi.q.bits : lo.q.bits);
+  bool done = false;
+  if (rows >= 8192) {
+    done = true;
+    if (C == 32) launch_ln_g<1, 4>(hi, lo, st);
+    else if (C == 64) launch_ln_g<2, 4>(hi, lo, st);
+    else if (C == 96) launch_ln_g<3, 4>(hi, lo, st);
+    else if (C == 128) launch_ln_g<4, 4>(hi, lo, st);
+    else if (C == 192 && min_bits * 4 >= 8) launch_ln_g<6, 8>(hi, lo, st);
+    else if (C == 256 && min_bits * 4 >= 8) launch_ln_g<8, 8>(hi, lo, st);
+    else done = false;
+  }
+  if (done) { ++g_launches; return; }
   switch (C / 32) {
     MIXAQ_LN_CASE(1, 8) MIXAQ_LN_CASE(2, 8) MIXAQ_LN_CASE(3, 8) MIXAQ_LN_CASE(4, 8) MIXAQ_LN_CASE(6, 4)
     MIXAQ_LN_CASE(8, 4) MIXAQ_LN_CASE(12, 2) MIXAQ_LN_CASE(16, 2) MIXAQ_LN_CASE(24, 1) MIXAQ_LN_CASE(32, 1)
