@@ -160,7 +160,7 @@ NUM_SMS, LANES_PER_SM = 148, 128
 TENSOR_CATS = {"gemm_qkv", "gemm_proj", "gemm_fc1_gelu", "gemm_fc2_scatter", "gemm_merge"}
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None
 # (stage-1 launch of the category, the largest of its 12 launches per step; profiles/gemm_tc_stage1_ncu_full.md)
-NCU_TRAFFIC_PER_LAUNCH = {"gemm_fc1_gelu": 5.03e6, "gemm_fc2_scatter": 47.5e6, "gemm_qkv": 5.02e6, "gemm_proj": 31.2e6}
+NCU_TRAFFIC_PER_LAUNCH = {"gemm_fc1_gelu": 5.03e6, "gemm_fc2_scatter": 47.1e6, "gemm_qkv": 5.01e6, "gemm_proj": 31.1e6}
 
 
 def run_ours(args):
