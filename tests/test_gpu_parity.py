@@ -126,6 +126,26 @@ def test_block_single_window_and_wide_dims(orc, mq, ctx):
         run_block_case(orc, mq, ctx, blk, synth.input_blobs(dim + 1, 1, 14, 15, dim, bg_std=0.5), 0.5)
 
 
+def test_block_random_shapes_and_settings(orc, mq, ctx):
+    """Seeded random sweep: widths, map sizes (ragged), batch, shift, bit-width pairs, ratios, pruning, bias sharing,
+    worst-case order.  Every case compares selection, all taps and the output bit for bit."""
+    rng = np.random.default_rng(2024)
+    dims = [32, 64, 96, 128, 192, 256]
+    bit_pairs = [(8, 4), (8, 8), (4, 2), (4, 4), (8, 2), (2, 2)]
+    for case in range(14):
+        dim = int(rng.choice(dims))
+        B = int(rng.integers(1, 4))
+        H, W = int(rng.integers(3, 30)), int(rng.integers(3, 30))
+        shift = int(rng.choice([0, 3, 1, 6]))
+        hb, lb = bit_pairs[int(rng.integers(len(bit_pairs)))]
+        low = float(rng.choice([0.0, 0.1, 0.3, 0.5, 0.8, 1.0]))
+        prune = float(rng.choice([0.0, 0.0, 0.2, 0.5]))
+        blk = synth.make_block(rng, dim, dim // 32, shift, int(rng.choice([4, 8])), hb, lb,
+                               share_bias=bool(rng.integers(2)))
+        x = synth.input_blobs(int(rng.integers(1 << 30)), B, H, W, dim, bg_std=0.5, gain=4.0)
+        run_block_case(orc, mq, ctx, blk, x, low, prune, reverse=bool(rng.integers(2)), stage_energy=bool(rng.integers(2)))
+
+
 def test_merge_parity(orc, mq, ctx):
     for (C, B, H, W) in [(32, 2, 9, 11), (96, 1, 20, 34), (192, 1, 13, 8)]:
         m = synth.make_merge(np.random.default_rng(C), C, 4, 8)
