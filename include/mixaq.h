@@ -121,6 +121,14 @@ const char*  mixaq_last_error(const mixaq_ctx* ctx);
 /* Reads the device status word (synchronises `cuda_stream`): MIXAQ_OK or MIXAQ_DEVICE_TIMEOUT. */
 mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream);
 
+/* Clears the status word (asynchronous on the stream). */
+mixaq_status mixaq_clear_device_status(mixaq_ctx* ctx, void* cuda_stream);
+/* Self-test of the failure path: launches one tiny CTA that waits, with the kernels' bounded wait, on a barrier that
+ * nothing signals.  The wait runs out after about a millisecond, the CTA raises the status word and returns normally;
+ * mixaq_last_device_status then reports MIXAQ_DEVICE_TIMEOUT and the context stays usable (clear the word with
+ * mixaq_clear_device_status).  No copy engine, tensor memory or invalid access is involved. */
+mixaq_status mixaq_selftest_wait_timeout(mixaq_ctx* ctx, void* cuda_stream);
+
 /* ---- the one definition of "how many windows does a ratio take out of n": floor(ratio*n + 1e-6) ---- */
 int          mixaq_low_count(float ratio, int n);
 /* counts[3] = {n_hi, n_lo, n_pr} per image for an H x W map: n_pr = cnt(prune, nW), n_lo = cnt(low, nW-n_pr). */

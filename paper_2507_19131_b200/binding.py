@@ -23,7 +23,7 @@ EXPORTS = [
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
-    "mixaq_norm_forward",
+    "mixaq_norm_forward", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -152,6 +152,12 @@ class Context:
 
     def set_graph_cache(self, enabled: bool):
         self.check(lib().mixaq_set_graph_cache(self.h, 1 if enabled else 0), "set_graph_cache")
+
+    def clear_device_status(self):
+        self.check(lib().mixaq_clear_device_status(self.h, _stream_ptr()), "clear_device_status")
+
+    def selftest_wait_timeout(self):
+        self.check(lib().mixaq_selftest_wait_timeout(self.h, _stream_ptr()), "selftest_wait_timeout")
 
     def launch_count(self) -> int:
         return lib().mixaq_last_launch_count(self.h)

@@ -76,6 +76,7 @@ struct GemmArgs {
   GemmBranch br[2];
 };
 bool launch_gemm(const GemmArgs& g, cudaStream_t st);
+void launch_wait_probe(int* status, cudaStream_t st);   // self-test of the bounded wait (it must run out)
 bool gemm_init();   // once per device context, before the first launch
 
 // ---- fused window attention ----------------------------------------------------------------------

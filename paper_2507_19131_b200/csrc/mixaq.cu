@@ -263,6 +263,18 @@ mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream) {
   return h == 0 ? MIXAQ_OK : MIXAQ_DEVICE_TIMEOUT;
 }
 
+mixaq_status mixaq_clear_device_status(mixaq_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  if (cudaMemsetAsync(ctx->d_status, 0, sizeof(int), (cudaStream_t)cuda_stream) != cudaSuccess) return check_cuda(ctx, "clear status");
+  return MIXAQ_OK;
+}
+
+mixaq_status mixaq_selftest_wait_timeout(mixaq_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  launch_wait_probe(ctx->d_status, (cudaStream_t)cuda_stream);
+  return check_cuda(ctx, "selftest_wait_timeout");
+}
+
 int mixaq_profile_categories(void) { return PC_COUNT; }
 const char* mixaq_profile_category_name(int cat) { return (cat >= 0 && cat < PC_COUNT) ? kProfNames[cat] : ""; }
 

@@ -279,6 +279,24 @@ def test_image_to_normed_stage_maps_end_to_end(orc, mq, ctx):
         assert np.array_equal(gg, ww)
 
 
+def test_bounded_wait_runs_out_and_the_context_stays_usable(orc, mq):
+    """Failure path without a fault: a barrier that nothing signals makes the kernels' bounded wait run out; the status
+    word reports it, can be cleared, and the next forward on the same context is correct."""
+    c = mq.Context(0)
+    try:
+        assert c.device_status() == 0
+        c.selftest_wait_timeout()
+        assert c.device_status() == -5                       # MIXAQ_DEVICE_TIMEOUT
+        c.clear_device_status()
+        assert c.device_status() == 0
+        blk = synth.make_block(np.random.default_rng(50), 32, 1, 3, 8, 8, 4)
+        x = synth.input_blobs(51, 1, 14, 15, 32, bg_std=0.5)
+        run_block_case(orc, mq, c, blk, x, 0.5)
+        assert c.device_status() == 0
+    finally:
+        c.close()
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
     import ctypes as C
     blk = synth.make_block(np.random.default_rng(40), 32, 1, 0, 8, 8, 4)
