@@ -18,7 +18,7 @@
  *     one exception: `prepared` buffers are read by every later forward call that gets the same params.
  *   - Feature maps are [B][H][W][C] binary32, channels contiguous.  C must be a multiple of 32, C/heads
  *     must be 32, window must be 7, hidden must be a multiple of 32.
- *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*); they allocate nothing and do
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*); they allocate no device memory and do
  *     not synchronise.  Errors found on the host are returned before anything is launched.
  *   - Activation codes are unsigned, `bits` in {8, 4, 2}.  Sub-byte codes are stored bit-packed, little end
  *     first: element e of a row lives in byte e*bits/8 at bit (e*bits) mod 8.
@@ -113,7 +113,8 @@ typedef struct {
 } mixaq_backbone_params;
 
 /* ---- context ---- */
-/* Creates a context on `device` (makes it current).  Holds the status word and cached TMA descriptors. */
+/* Creates a context on `device` (makes it current).  Holds the status word, the captured graphs of
+ * mixaq_backbone_forward and the profiling events. */
 mixaq_status mixaq_create(mixaq_ctx** ctx, int device);
 mixaq_status mixaq_destroy(mixaq_ctx* ctx);
 /* Text of the last host-side error of this context (static storage, valid until the next call). */

@@ -1,6 +1,7 @@
 // Memory-bound row kernels: gather + LayerNorm + quantize + bit-pack (both branches in one launch),
 // the patch-merging gather, and the pass-through copy of pruned windows (MixA-Q Section 3.2 / 3.4).
-// One warp owns one token row; lane l holds channels l, l+32, l+64, ... so every load is a full 128-byte line.
+// Two LayerNorm kernels with the same summation tree: one warp per row (lane l holds channels l, l+32, l+64, ...,
+// every load a full 128-byte line) and, for large batches of narrow rows, 4 or 8 lanes per row with vector loads.
 #include "kernels.h"
 
 namespace mixaq {
