@@ -8,11 +8,11 @@
 //               128-byte-swizzled K-major stages (cp.async.bulk.tensor, no multicast), completion on mbarriers;
 //   warp 1      MMA issuer: one thread feeds the tensor core; the accumulator alternates between two TMEM
 //               buffers so that the epilogue of tile i overlaps the loads and MMAs of tile i+1;
-//   warps 2-3   unpack producers for 4-bit / 2-bit branches: the bit-packed rows of the k-block arrive by TMA in a
+//   warps 2-5   unpack producers for 4-bit / 2-bit branches: the bit-packed rows of the k-block arrive by TMA in a
 //               staging slot of the stage; these warps expand them to one code per byte, shared to shared, into
 //               the swizzled layout (rows whose byte pitch is no multiple of 16 cannot be described to the TMA
 //               unit and are read with plain loads instead);
-//   warps 4-..  epilogue (16 warps for the code outputs, 8 for the binary32 outputs): tcgen05.ld (one row per thread, 16 columns per load) + the fused epilogue of the mode.
+//   then        epilogue (12 warps for the code outputs, 8 for the binary32 outputs): tcgen05.ld (one row per thread, 16 columns per load) + the fused epilogue of the mode.
 // Every wait on an mbarrier is bounded; on expiry the CTA raises the status word, drains, frees its tensor
 // memory and returns.
 #include <cuda.h>
@@ -26,15 +26,15 @@ constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int BK = 128;            // codes (bytes) per row and stage = one 128-byte swizzle row
 constexpr int UMMA_K = 32;         // codes per tcgen05.mma kind::i8
 constexpr int A_STAGE_BYTES = BM * BK;
-constexpr int NUM_UNPACK_WARPS = 2;            // warps 2..3
-constexpr int NUM_UNPACK_THREADS = NUM_UNPACK_WARPS * 32;
-constexpr int MAX_EPI_WARPS = 16;              // warps 4.. : 16 for the arithmetic-bound code epilogues, 8 for the binary32 ones
-__host__ __device__ constexpr int epi_warps(int mode) { return (mode == EPI_QKV || mode == EPI_FC1) ? 16 : 8; }
+// warps 2..5 expand sub-byte codes (two warps left the long-K main loops of 4-bit tiles waiting for the expansion;
+// eight cost more registers than they return)
+__host__ __device__ constexpr int unpack_warps(int mode) { return 4; }
+constexpr int MAX_EPI_WARPS = 16;              // epilogue warps: 12 for the arithmetic-bound code epilogues, 8 for the binary32 ones
+__host__ __device__ constexpr int epi_warps(int mode) { return (mode == EPI_QKV || mode == EPI_FC1) ? 12 : 8; }
 constexpr int MAX_BN = 256;
 constexpr int EPI_WARP_COLS = MAX_BN / 2;      // most columns one epilogue warp handles per tile (two warps per lane quarter)
 constexpr int MAX_RING = 6;
 constexpr uint32_t MAX_POLLS = 1u << 20;       // tries per wait; each try may sleep up to WAIT_HINT_NS
-constexpr int UNPACK_ITEMS = BM * (BK / UMMA_K) / NUM_UNPACK_THREADS;   // (row, 32-code group) items per thread and stage
 
 struct TcParams {
   GemmArgs g;
@@ -132,7 +132,7 @@ __device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int t) {
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(128 + 32 * epi_warps(MODE), 1)
+__global__ void __launch_bounds__(32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
           const __grid_constant__ CUtensorMap tmB, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -150,6 +150,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   constexpr int NUM_EPI_WARPS = epi_warps(MODE);
+  constexpr int NUM_UNPACK_WARPS = unpack_warps(MODE), NUM_UNPACK_THREADS = NUM_UNPACK_WARPS * 32;
+  constexpr int FIRST_EPI_WARP = 2 + NUM_UNPACK_WARPS;
+  constexpr int UNPACK_ITEMS = BM * (BK / UMMA_K) / NUM_UNPACK_THREADS;   // (row, 32-code group) items per thread and stage
   constexpr int EPI_SPLIT = NUM_EPI_WARPS / 4;   // warps that share a TMEM lane quarter deal its chunks round-robin
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int K = p.g.K;
@@ -242,9 +245,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
       }
     }
     __syncwarp();
-  } else if (warp < 4) {
+  } else if (warp < FIRST_EPI_WARP) {
     // ---- unpack producers: bit-packed rows -> one code per byte, written in the swizzled layout ----
-    const int ptid = tid - 64;                   // 0..63
+    const int ptid = tid - 64;                   // 0 .. NUM_UNPACK_THREADS-1
     int it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
@@ -264,7 +267,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           const uint8_t* sp = sa + A_STAGE_BYTES + p.BN * BK;
           const int kgroups = min(BK, K - kb * BK) / UMMA_K;
-          // item i of this thread: row r = (ptid + 64*i) / 4, 32-code group kg = (ptid + 64*i) % 4
+          // item i of this thread: row r = item / 4, 32-code group kg = item % 4, item = ptid + NUM_UNPACK_THREADS * i
 #pragma unroll
           for (int i = 0; i < UNPACK_ITEMS; ++i) {
             const int item = ptid + NUM_UNPACK_THREADS * i;
@@ -294,7 +297,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     __syncwarp();
   } else {
     // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).. and takes every EPI_SPLIT-th 16-column chunk ----
-    const int e = warp - 4, q = warp & 3, sub = e >> 2;
+    const int e = warp - FIRST_EPI_WARP, q = warp & 3, sub = e >> 2;   // any 4 consecutive warps cover the 4 lane quarters
     float* stage = s_stage + e * EPI_STAGE_FLOATS;
     int32_t* c_zc = s_consts + e * 3 * EPI_WARP_COLS;
     float* c_mult = reinterpret_cast<float*>(c_zc + EPI_WARP_COLS);
@@ -455,7 +458,7 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles)
   int grid = p.total_tiles < sms ? p.total_tiles : sms;
   if (grid > p.n_tiles && grid < p.total_tiles) grid -= grid % p.n_tiles;
-  k_gemm_tc<MODE><<<grid, 128 + 32 * epi_warps(MODE), smem, st>>>(mA[0], mA[1], mB, p);
+  k_gemm_tc<MODE><<<grid, 32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), smem, st>>>(mA[0], mA[1], mB, p);
   ++g_launches;
   return true;
 }
