@@ -55,6 +55,8 @@ def check_taps(orc, blk, ref, got, counts):
 
 
 def run_block_case(orc, mq, ctx, blk, x, low, prune=0.0, reverse=False, stage_energy=False, taps=True):
+    # the C ABI takes the ratios as binary32: both sides get exactly that value (0.11f * 6000 is below 660)
+    low, prune = float(F32(low)), float(F32(prune))
     db = mq.DeviceBlock(ctx, blk)
     xd = dev(x)
     e_ref = e_dev = None
@@ -144,6 +146,20 @@ def test_block_random_shapes_and_settings(orc, mq, ctx):
                                share_bias=bool(rng.integers(2)))
         x = synth.input_blobs(int(rng.integers(1 << 30)), B, H, W, dim, bg_std=0.5, gain=4.0)
         run_block_case(orc, mq, ctx, blk, x, low, prune, reverse=bool(rng.integers(2)), stage_energy=bool(rng.integers(2)))
+
+
+def test_many_windows_per_image_and_the_limit(orc, mq, ctx):
+    """A long thin map with 6000 windows in one image (the ranking holds one image's scores in shared memory; the
+    limit is 6144 windows), and a map beyond the limit, which must be refused before anything is launched."""
+    blk = synth.make_block(np.random.default_rng(60), 32, 1, 3, 8, 8, 4)
+    x = synth.input_student_t(61, 1, 7, 7 * 6000, 32)
+    run_block_case(orc, mq, ctx, blk, x, 0.37, 0.11, taps=False)
+    db = mq.DeviceBlock(ctx, blk)
+    big = torch.zeros((1, 7, 7 * 6200, 32), device="cuda")
+    with pytest.raises(mq.MixaqError) as e:
+        mq.block_forward(ctx, db, big, 0.5)
+    assert e.value.status == -2
+    assert ctx.device_status() == 0
 
 
 def test_merge_parity(orc, mq, ctx):
