@@ -367,6 +367,14 @@ def run_ours(args):
                 "note": "800x1333x3 image -> 200x334x96 tokens (3 launches); LayerNorm of the 4 stage maps (4 launches); "
                         "stream launches, not part of `value`"}
 
+    # tensor-core issue rate as the library's own MMA loop reaches it (context for the tensor fractions above)
+    mma_peak = None
+    if world == 1:
+        mma_peak = {"kind_i8_tops": round(ctx.measure_mma_peak(0, 8000), 1),
+                    "kind_f8f6f4_e4m3_tops": round(ctx.measure_mma_peak(1, 8000), 1),
+                    "note": "all SMs issue 128x256x32 tcgen05.mma from shared memory into TMEM; f8f6f4 is the path that "
+                            "carries 4/6-bit operand formats: it is not faster than i8, so no narrower MMA path is used"}
+
     status = ctx.device_status()
     if rank != 0:
         if world > 1:
@@ -395,6 +403,7 @@ def run_ours(args):
         "low_ratio_sweep_images_per_sec": sweep,
         "paper_cost_model": cost,
         "stem_and_norms": stem,
+        "mma_issue_rate": mma_peak,
         "device_status": status,
     }
     if args.cpu_baseline and world == 1:

@@ -217,6 +217,15 @@ mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled);
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 
+/* ---- tensor-core issue rate as this library reaches it (the denominator for the GEMMs' tensor-pipe fraction):
+ *      all SMs at once issue `groups` x 4 tcgen05.mma of 128 x 256 x 32 from shared-memory operands into TMEM.
+ *      kind 0: kind::i8 (u8 x s8 -> s32), the path the GEMMs use.  kind 1: kind::f8f6f4 with E4M3 operands, the path
+ *      that also carries the 4-bit and 6-bit operand formats (in 8-bit containers): its rate bounds what a narrower
+ *      operand type could give.  `scratch`: >= 8 KiB of device memory.  Synchronises the stream; result in 10^12
+ *      operations (2 per multiply-accumulate) per second. ---- */
+mixaq_status mixaq_measure_mma_peak(mixaq_ctx* ctx, int kind, int groups, void* scratch, size_t scratch_bytes,
+                                    double* tera_ops_per_s, void* cuda_stream);
+
 /* ---- per-kernel timing (the paper reports no time breakdown; this is the library's own tracing aid).
  *      Between begin and end every kernel family launched through this context is bracketed by CUDA events on
  *      the launching stream.  end() synchronises the stream and returns, per category (see

@@ -23,7 +23,7 @@ EXPORTS = [
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
-    "mixaq_norm_forward", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout",
+    "mixaq_norm_forward", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -158,6 +158,14 @@ class Context:
 
     def selftest_wait_timeout(self):
         self.check(lib().mixaq_selftest_wait_timeout(self.h, _stream_ptr()), "selftest_wait_timeout")
+
+    def measure_mma_peak(self, kind: int = 0, groups: int = 2000) -> float:
+        """Tensor-core issue rate in TOP/s (kind 0: kind::i8; 1: kind::f8f6f4 with E4M3 operands)."""
+        scratch = torch.empty(8192, dtype=torch.uint8, device=self.device)
+        out = C.c_double()
+        self.check(lib().mixaq_measure_mma_peak(self.h, kind, groups, _ptr(scratch), C.c_size_t(8192), C.byref(out),
+                                                _stream_ptr()), "measure_mma_peak")
+        return float(out.value)
 
     def launch_count(self) -> int:
         return lib().mixaq_last_launch_count(self.h)

@@ -483,6 +483,80 @@ void launch_wait_probe(int* status, cudaStream_t st) {
   ++g_launches;
 }
 
+// Issue-rate microbenchmark of the tensor core: every CTA (one per SM) keeps a 128 x 128-byte A tile and a
+// 256 x 128-byte B tile in shared memory and issues `groups` x 4 MMAs of 128 x 256 x 32 into one TMEM accumulator,
+// then waits (bounded) for the commit.  KIND 0: kind::i8 (u8 x s8 -> s32), the path the GEMMs use.
+// KIND 1: kind::f8f6f4 with E4M3 operands (-> f32); this is also the path that carries 4-bit and 6-bit operand
+// formats on sm_100a (in 8-bit shared-memory containers), so its rate bounds what a narrower operand type could give.
+template <int KIND>
+__global__ void __launch_bounds__(128, 1) k_mma_peak(int groups, unsigned long long* ns_out, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  uint64_t* bar = reinterpret_cast<uint64_t*>(smem + A_STAGE_BYTES + MAX_BN * BK);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar + 1);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  for (int i = tid; i < (A_STAGE_BYTES + MAX_BN * BK) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem)[i] = ((uint32_t)(i * 37 + 11) * 0x01010101u) & 0x3E3E3E3Eu;   // finite in E4M3 too
+  if (tid == 0) { mbar_init(smem_u32(bar), 1u); asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+  if (tid == 0) {
+    // instruction descriptor: D format (s32 = 2 / f32 = 1) at bit 4, A format at 7, B format at 10, N/8 at 17, M/16 at 24
+    const uint32_t idesc = KIND == 0 ? ((2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(MAX_BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24))
+                                     : ((1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(MAX_BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24));
+    const uint64_t adesc = smem_desc_sw128(base), bdesc = smem_desc_sw128(base + A_STAGE_BYTES);
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    for (int g = 0; g < groups; ++g)
+      for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+        const uint32_t accumulate = (g > 0 || kk > 0) ? 1u : 0u;
+        if (KIND == 0) {
+          mma_i8(tmem_base, adesc + (uint64_t)(kk * (UMMA_K >> 4)), bdesc + (uint64_t)(kk * (UMMA_K >> 4)), idesc, accumulate);
+        } else {
+          asm volatile(
+              "{\n\t.reg .pred p;\n\t"
+              "setp.ne.b32 p, %4, 0;\n\t"
+              "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+              ::"r"(tmem_base), "l"(adesc + (uint64_t)(kk * (UMMA_K >> 4))), "l"(bdesc + (uint64_t)(kk * (UMMA_K >> 4))),
+                "r"(idesc), "r"(accumulate) : "memory");
+        }
+      }
+    mma_commit(smem_u32(bar));
+    bool done = false;
+    for (uint32_t it = 0; it < MAX_POLLS && !done; ++it) done = mbar_try_wait(smem_u32(bar), 0);
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+    if (!done) atomicExch(status, 1);
+    ns_out[blockIdx.x] = t1 - t0;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+}
+
+// ns_out: one entry per SM (device memory).  Returns the grid size, 0 on failure.
+int launch_mma_peak(int kind, int groups, unsigned long long* ns_out, int* status, cudaStream_t st) {
+  const int sms = num_sms();
+  const size_t smem = A_STAGE_BYTES + MAX_BN * BK + 1024 + 64;
+  if (kind == 0) {
+    if (cudaFuncSetAttribute(k_mma_peak<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+    k_mma_peak<0><<<sms, 128, smem, st>>>(groups, ns_out, status);
+  } else {
+    if (cudaFuncSetAttribute(k_mma_peak<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+    k_mma_peak<1><<<sms, 128, smem, st>>>(groups, ns_out, status);
+  }
+  ++g_launches;
+  return sms;
+}
+
 // One-time set-up per device context (kept out of the launch path so that launches can be stream-captured):
 // opt-in to large dynamic shared memory for every epilogue mode, resolve the tensor-map encoder, read the SM count.
 bool gemm_init() {

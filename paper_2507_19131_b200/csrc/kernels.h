@@ -77,6 +77,8 @@ struct GemmArgs {
 };
 bool launch_gemm(const GemmArgs& g, cudaStream_t st);
 void launch_wait_probe(int* status, cudaStream_t st);   // self-test of the bounded wait (it must run out)
+// tensor-core issue-rate microbenchmark (kind 0: i8, 1: f8f6f4/E4M3); ns per SM into ns_out; returns the grid size
+int launch_mma_peak(int kind, int groups, unsigned long long* ns_out, int* status, cudaStream_t st);
 bool gemm_init();   // once per device context, before the first launch
 
 // ---- fused window attention ----------------------------------------------------------------------

@@ -275,6 +275,25 @@ mixaq_status mixaq_selftest_wait_timeout(mixaq_ctx* ctx, void* cuda_stream) {
   return check_cuda(ctx, "selftest_wait_timeout");
 }
 
+mixaq_status mixaq_measure_mma_peak(mixaq_ctx* ctx, int kind, int groups, void* scratch, size_t scratch_bytes,
+                                    double* tera_ops_per_s, void* cuda_stream) {
+  if (!ctx || !scratch || !tera_ops_per_s || groups <= 0 || (kind != 0 && kind != 1)) return MIXAQ_INVALID_ARG;
+  if (scratch_bytes < 1024 * sizeof(unsigned long long)) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "mma peak: scratch of 8 KiB needed");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  unsigned long long* d_ns = (unsigned long long*)scratch;
+  const int sms = launch_mma_peak(kind, groups, d_ns, ctx->d_status, st);
+  if (sms <= 0 || sms > 1024) return check_cuda(ctx, "mma peak") == MIXAQ_OK ? MIXAQ_INTERNAL : MIXAQ_CUDA_ERROR;
+  std::vector<unsigned long long> ns(sms);
+  if (cudaMemcpyAsync(ns.data(), d_ns, sizeof(unsigned long long) * sms, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) return check_cuda(ctx, "mma peak");
+  unsigned long long worst = 1;
+  for (auto v : ns) worst = v > worst ? v : worst;
+  // every SM issued groups x 4 MMAs of 128 x 256 x 32 multiply-accumulates; all SMs ran at once: the slowest one counts
+  const double ops = 2.0 * 128.0 * 256.0 * 32.0 * 4.0 * (double)groups * (double)sms;
+  *tera_ops_per_s = ops / ((double)worst * 1e-9) / 1e12;
+  return check_cuda(ctx, "mma peak");
+}
+
 int mixaq_profile_categories(void) { return PC_COUNT; }
 const char* mixaq_profile_category_name(int cat) { return (cat >= 0 && cat < PC_COUNT) ? kProfNames[cat] : ""; }
 

@@ -331,6 +331,16 @@ def test_calibration_on_the_gpu_feeds_the_quantized_forward(orc, mq, ctx):
         assert np.array_equal(g.cpu().numpy(), w)
 
 
+def test_mma_issue_rate_microbenchmark(mq, ctx):
+    """The library's own tensor-core loop: kind::i8 reaches petaops, and kind::f8f6f4 (the path of the 4/6-bit operand
+    formats) is not faster, which is why the low branch keeps using kind::i8."""
+    i8 = ctx.measure_mma_peak(0, 2000)
+    f8 = ctx.measure_mma_peak(1, 2000)
+    assert ctx.device_status() == 0
+    assert 1500.0 < i8 < 6000.0 and 1500.0 < f8 < 6000.0
+    assert f8 < 1.1 * i8
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
     import ctypes as C
     blk = synth.make_block(np.random.default_rng(40), 32, 1, 0, 8, 8, 4)
