@@ -20,9 +20,13 @@ __global__ void __launch_bounds__(256) k_energy(const float* __restrict__ x, int
   int e = 0;
   if (tok < ntok) {
     const float4* row = reinterpret_cast<const float4*>(x + tok * C);
-    for (int c4 = sub; c4 < C / 4; c4 += 8) {
-      const float4 v = __ldg(row + c4);
-      e += score_code_sq(v.x, inv) + score_code_sq(v.y, inv) + score_code_sq(v.z, inv) + score_code_sq(v.w, inv);
+    for (int c0 = sub; c0 < C / 4; c0 += 32) {          // four loads in flight per lane
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = c0 + 8 * u < C / 4 ? __ldg(row + c0 + 8 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        e += score_code_sq(v[u].x, inv) + score_code_sq(v[u].y, inv) + score_code_sq(v[u].z, inv) + score_code_sq(v[u].w, inv);
     }
   }
 #pragma unroll
