@@ -562,7 +562,7 @@ void orc_patch_embed(const orc_embed* e, const float* img, int B, int Hi, int Wi
 
 void orc_backbone_forward(int num_stages, const int* depths, const orc_block* blocks, const orc_merge* merges,
                           const float* x0, float* const* stage_out, int B, int H0, int W0,
-                          const double* low_ratio_per_pair, const double* prune_ratio_per_pair) {
+                          const double* low_ratio_per_pair, const double* prune_ratio_per_pair, int allow_elevation) {
   int H = H0, W = W0, blk = 0;
   std::vector<float> cur, nxt;
   for (int s = 0; s < num_stages; ++s) {
@@ -578,11 +578,19 @@ void orc_backbone_forward(int num_stages, const int* depths, const orc_block* bl
     // importance is computed once per stage, before its first block, and shared (Section 3.2)
     std::vector<int32_t> energy((size_t)B * H * W);
     orc_energy(cur.data(), B, H, W, C, blocks[blk].score_inv_scale, energy.data());
+    // Windows keep their precision class within a stage (Section 4.4, "Windows Elevation": letting compressed windows
+    // return to high precision in later blocks is the ablation, not the default): a pair's effective ratios are the
+    // largest ratios of the pairs of this stage so far, so the set of non-high windows never shrinks.
+    double low_eff = 0.0, prune_eff = 0.0;
     for (int i = 0; i < depths[s]; ++i, ++blk) {
       int pair = blk / 2;
+      double lr = low_ratio_per_pair[pair], pr = prune_ratio_per_pair ? prune_ratio_per_pair[pair] : 0.0;
+      if (!allow_elevation) {
+        low_eff = std::max(low_eff, lr); prune_eff = std::max(prune_eff, pr);
+        lr = low_eff; pr = prune_eff;
+      }
       nxt.resize(cur.size());
-      orc_block_forward(&blocks[blk], cur.data(), nxt.data(), B, H, W, low_ratio_per_pair[pair],
-                        prune_ratio_per_pair ? prune_ratio_per_pair[pair] : 0.0, energy.data(), 0,
+      orc_block_forward(&blocks[blk], cur.data(), nxt.data(), B, H, W, lr, pr, energy.data(), 0,
                         nullptr, nullptr, nullptr, nullptr, nullptr);
       cur.swap(nxt);
     }

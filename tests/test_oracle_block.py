@@ -376,3 +376,28 @@ def test_patch_embed_quantized_from_pinned_primitives_and_onehot(orc):
     deq = orc.dequantize(codes[:, :32], e2.aq)
     want2 = orc.layernorm(deq, e2.ln_g, e2.ln_b)
     assert np.array_equal(g2, want2)
+
+
+# ------------------------------------------------------------------------------------------------
+# precision classes within a stage (Section 4.4, "Windows Elevation")
+# ------------------------------------------------------------------------------------------------
+def test_no_elevation_keeps_classes_within_a_stage(orc):
+    """One stage of three pairs whose ratios go down and up.  Default: a pair's effective ratio is the largest ratio so
+    far in the stage (compressed windows stay compressed), so the forward equals the one with the running-maximum
+    ratios; with elevation allowed every pair uses its own ratio."""
+    bb = synth.make_backbone(9, [32], [6], [1], 8, 8, 4)
+    x = synth.input_blobs(10, 1, 21, 28, 32, bg_std=0.5, gain=4.0)
+    ratios = [0.5, 0.2, 0.4]
+    dflt = orc.backbone_forward(bb, x, ratios)[0]
+    runmax = orc.backbone_forward(bb, x, [0.5, 0.5, 0.5], allow_elevation=True)[0]
+    elev = orc.backbone_forward(bb, x, ratios, allow_elevation=True)[0]
+    assert np.array_equal(dflt, runmax)
+    assert not np.array_equal(dflt, elev)
+    # non-decreasing ratios: both policies agree
+    up = [0.1, 0.3, 0.6]
+    assert np.array_equal(orc.backbone_forward(bb, x, up)[0], orc.backbone_forward(bb, x, up, allow_elevation=True)[0])
+    # the running maximum does not leak into the next stage
+    bb2 = synth.make_backbone(11, [32, 64], [2, 2], [1, 2], 8, 8, 4)
+    a = orc.backbone_forward(bb2, x, [0.6, 0.1])
+    b = orc.backbone_forward(bb2, x, [0.6, 0.1], allow_elevation=True)
+    assert all(np.array_equal(u, v) for u, v in zip(a, b))
