@@ -214,6 +214,12 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
  * enabled = 0 switches the cache off and drops the stored graphs; it is on by default. */
 mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled);
 
+/* Within a stage windows keep their precision class (Section 4.4, "Windows Elevation": letting compressed windows
+ * return to high precision in later blocks is the paper's ablation, not its default).  mixaq_backbone_forward
+ * therefore uses, for every block pair, the largest low-bit ratio and the largest prune ratio of the stage's pairs so
+ * far, so the set of non-high windows never shrinks inside a stage.  allow = 1 makes every pair use its own ratios. */
+mixaq_status mixaq_set_window_elevation(mixaq_ctx* ctx, int allow);
+
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 

@@ -28,6 +28,7 @@ struct mixaq_ctx {
   char err[256];
   bool profiling;
   bool graph_cache;                    // replay backbone forwards as CUDA graphs (see mixaq_set_graph_cache)
+  bool allow_elevation;                // backbone: every pair uses its own ratios even if an earlier pair of the stage had larger ones
   std::vector<GraphEntry> graphs;
   std::vector<ProfRec> prof;          // event pairs recorded since mixaq_profile_begin
   std::vector<cudaEvent_t> pool;      // events ready for reuse
@@ -231,7 +232,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
       !gemm_init()) {
     cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
@@ -638,6 +639,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     const char has_prune = prune_ratio_per_pair ? 1 : 0; put(&has_prune, 1);
     if (prune_ratio_per_pair) put(prune_ratio_per_pair, sizeof(float) * npairs);
     put(&workspace, sizeof(workspace)); put(&workspace_bytes, sizeof(workspace_bytes)); put(&st, sizeof(st));
+    const char elev = ctx->allow_elevation ? 1 : 0; put(&elev, 1);
     for (auto& g : ctx->graphs)
       if (g.key == key) {
         if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return check_cuda(ctx, "backbone_forward (graph launch)");
@@ -669,8 +671,17 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     const size_t sel_stride = carve_sel(B, H, W, nullptr).bytes;
     std::vector<SelWs> sels(d);
     std::vector<SelectArgs> sargs(d);
+    // Windows keep their precision class within a stage (Section 4.4, "Windows Elevation"): unless elevation is
+    // allowed, a pair's effective ratios are the largest ratios of the stage's pairs so far.
+    std::vector<float> lr_eff(d), pr_eff(d);
+    float lmax = 0.f, pmax = 0.f;
     for (int i = 0; i < d; ++i) {
-      const float lr = low_ratio_per_pair[(blk + i) / 2], pr = prune_ratio_per_pair ? prune_ratio_per_pair[(blk + i) / 2] : 0.f;
+      float lr = low_ratio_per_pair[(blk + i) / 2], pr = prune_ratio_per_pair ? prune_ratio_per_pair[(blk + i) / 2] : 0.f;
+      if (!ctx->allow_elevation) { lmax = std::max(lmax, lr); pmax = std::max(pmax, pr); lr = lmax; pr = pmax; }
+      lr_eff[i] = lr; pr_eff[i] = pr;
+    }
+    for (int i = 0; i < d; ++i) {
+      const float lr = lr_eff[i], pr = pr_eff[i];
       Geometry g = geometry(H, W, lr, pr);
       if ((size_t)g.nW * 8 > 48 * 1024) { result = fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many windows per image (max 6144)"); break; }
       sels[i] = carve_sel(B, H, W, ws.sel + (size_t)i * sel_stride);
@@ -682,8 +693,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     total += g_launches;
     for (int i = 0; i < d; ++i, ++blk) {
       float* dst = ((d - 1 - i) % 2 == 0) ? out_s : ws.scratch;
-      result = block_forward_impl(ctx, &p->blocks[blk], cur, dst, B, H, W, low_ratio_per_pair[blk / 2],
-                                  prune_ratio_per_pair ? prune_ratio_per_pair[blk / 2] : 0.f, nullptr, nullptr,
+      result = block_forward_impl(ctx, &p->blocks[blk], cur, dst, B, H, W, lr_eff[i], pr_eff[i], nullptr, nullptr,
                                   ws.block, ws.block_bytes, nullptr, &sels[i], st);
       if (result != MIXAQ_OK) break;
       total += ctx->launches;
@@ -789,6 +799,12 @@ mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float*
     return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "norm: unsupported C");
   ctx->launches = g_launches;
   return check_cuda(ctx, "norm_forward");
+}
+
+mixaq_status mixaq_set_window_elevation(mixaq_ctx* ctx, int allow) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  ctx->allow_elevation = allow != 0;
+  return MIXAQ_OK;
 }
 
 mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled) {

@@ -204,6 +204,37 @@ def test_backbone_graph_replay_reads_fresh_data(orc, mq, ctx):
     torch.cuda.current_stream().wait_stream(side)
 
 
+def test_precision_classes_within_a_stage_and_the_elevation_switch(orc, mq):
+    """A stage of three pairs with ratios that go down and up: default (classes kept: running maximum) and the
+    elevation ablation (every pair its own ratio), each against the oracle in the same mode; with and without the graph."""
+    bb = synth.make_backbone(9, [64], [6], [2], 8, 8, 4)
+    x = synth.input_blobs(10, 2, 21, 29, 64, bg_std=0.5, gain=4.0)
+    ratios, prunes = [0.5, 0.2, 0.4], [0.1, 0.3, 0.0]
+    c = mq.Context(0)
+    try:
+        dbb = mq.DeviceBackbone(c, bb, 2, 21, 29)
+        side = torch.cuda.Stream()
+        for allow in (False, True):
+            c.set_window_elevation(allow)
+            want = orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=allow)[0]
+            got = mq.backbone_forward(c, dbb, dev(x), ratios, prunes)[0].cpu().numpy()       # default stream: direct launches
+            assert np.array_equal(got, want), f"allow={allow}"
+            with torch.cuda.stream(side):
+                xd = dev(x)
+                for _ in range(2):                                                             # capture, then replay
+                    got = mq.backbone_forward(c, dbb, xd, ratios, prunes)[0]
+                side.synchronize()
+                assert np.array_equal(got.cpu().numpy(), want), f"graph, allow={allow}"
+        c.set_graph_cache(False)
+        with torch.cuda.stream(side):
+            got = mq.backbone_forward(c, dbb, dev(x), ratios, prunes)[0]
+            side.synchronize()
+        assert np.array_equal(got.cpu().numpy(), orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=True)[0])
+        assert c.device_status() == 0
+    finally:
+        c.close()
+
+
 def test_config2_stage1_pair_full_size(orc, mq, ctx):
     """Block pair at 200x334 (W-MSA then SW-MSA with mask), B=2, Student-t input, ratio 0.3, shared stage energy."""
     wl = synth.config2()
