@@ -220,6 +220,11 @@ mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled);
  * far, so the set of non-high windows never shrinks inside a stage.  allow = 1 makes every pair use its own ratios. */
 mixaq_status mixaq_set_window_elevation(mixaq_ctx* ctx, int allow);
 
+/* Worst-case window selection for mixaq_backbone_forward (Table 4: "importance in reverse order"): the LOWEST
+ * scores go to the high-precision branch in every block.  Off by default; the block call has the same switch in
+ * mixaq_select_opts. */
+mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse);
+
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 

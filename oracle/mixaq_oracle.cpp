@@ -562,7 +562,8 @@ void orc_patch_embed(const orc_embed* e, const float* img, int B, int Hi, int Wi
 
 void orc_backbone_forward(int num_stages, const int* depths, const orc_block* blocks, const orc_merge* merges,
                           const float* x0, float* const* stage_out, int B, int H0, int W0,
-                          const double* low_ratio_per_pair, const double* prune_ratio_per_pair, int allow_elevation) {
+                          const double* low_ratio_per_pair, const double* prune_ratio_per_pair, int allow_elevation,
+                          int reverse) {
   int H = H0, W = W0, blk = 0;
   std::vector<float> cur, nxt;
   for (int s = 0; s < num_stages; ++s) {
@@ -590,7 +591,7 @@ void orc_backbone_forward(int num_stages, const int* depths, const orc_block* bl
         lr = low_eff; pr = prune_eff;
       }
       nxt.resize(cur.size());
-      orc_block_forward(&blocks[blk], cur.data(), nxt.data(), B, H, W, lr, pr, energy.data(), 0,
+      orc_block_forward(&blocks[blk], cur.data(), nxt.data(), B, H, W, lr, pr, energy.data(), reverse,
                         nullptr, nullptr, nullptr, nullptr, nullptr);
       cur.swap(nxt);
     }

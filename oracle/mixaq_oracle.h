@@ -113,7 +113,8 @@ void  orc_merge_forward(const orc_merge* m, const float* x, int B, int H, int W,
 void  orc_backbone_forward(int num_stages, const int* depths, const orc_block* blocks, const orc_merge* merges,
                            const float* x0, float* const* stage_out, int B, int H0, int W0,
                            const double* low_ratio_per_pair, const double* prune_ratio_per_pair,
-                           int allow_elevation /* 0: classes are kept within a stage (the paper's default) */);
+                           int allow_elevation /* 0: classes are kept within a stage (the paper's default) */,
+                           int reverse /* 1: worst-case selection order (Table 4) in every block */);
 void  orc_patch_embed(const orc_embed* e, const float* img, int B, int Hi, int Wi, float* x0 /* [B][ceil(Hi/4)][ceil(Wi/4)][C0] */);
 void  orc_set_threads(int n);
 int   orc_get_threads(void);

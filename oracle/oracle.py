@@ -318,7 +318,7 @@ def merge_forward(m, x, quant=True):
     return y
 
 
-def backbone_forward(bb, x, low_ratios, prune_ratios=None, quant=True, allow_elevation=False):
+def backbone_forward(bb, x, low_ratios, prune_ratios=None, quant=True, allow_elevation=False, reverse=False):
     """bb: object with dims, depths, blocks, merges.  Returns the list of stage outputs."""
     x = np.ascontiguousarray(x, np.float32)
     B, H, W, _ = x.shape
@@ -338,7 +338,7 @@ def backbone_forward(bb, x, low_ratios, prune_ratios=None, quant=True, allow_ele
     pr = None
     if prune_ratios is not None:
         pr = (C.c_double * npairs)(*([float(r) for r in prune_ratios] + [0.0] * (npairs - len(prune_ratios))))
-    lib().orc_backbone_forward(ns, depths, blocks, merges, _p(x), ptrs, B, H, W, lr, pr, 1 if allow_elevation else 0)
+    lib().orc_backbone_forward(ns, depths, blocks, merges, _p(x), ptrs, B, H, W, lr, pr, 1 if allow_elevation else 0, 1 if reverse else 0)
     return outs
 
 

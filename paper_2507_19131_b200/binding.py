@@ -23,7 +23,7 @@ EXPORTS = [
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
-    "mixaq_norm_forward", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation",
+    "mixaq_norm_forward", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -149,6 +149,9 @@ class Context:
 
     def device_status(self) -> int:
         return lib().mixaq_last_device_status(self.h, _stream_ptr())
+
+    def set_reverse_selection(self, reverse: bool):
+        self.check(lib().mixaq_set_reverse_selection(self.h, 1 if reverse else 0), "set_reverse_selection")
 
     def set_window_elevation(self, allow: bool):
         self.check(lib().mixaq_set_window_elevation(self.h, 1 if allow else 0), "set_window_elevation")

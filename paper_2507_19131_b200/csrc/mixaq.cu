@@ -28,6 +28,7 @@ struct mixaq_ctx {
   char err[256];
   bool profiling;
   bool graph_cache;                    // replay backbone forwards as CUDA graphs (see mixaq_set_graph_cache)
+  bool reverse_selection;              // backbone: worst-case selection order (Table 4) in every block
   bool allow_elevation;                // backbone: every pair uses its own ratios even if an earlier pair of the stage had larger ones
   std::vector<GraphEntry> graphs;
   std::vector<ProfRec> prof;          // event pairs recorded since mixaq_profile_begin
@@ -232,7 +233,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
       !gemm_init()) {
     cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
@@ -639,7 +640,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     const char has_prune = prune_ratio_per_pair ? 1 : 0; put(&has_prune, 1);
     if (prune_ratio_per_pair) put(prune_ratio_per_pair, sizeof(float) * npairs);
     put(&workspace, sizeof(workspace)); put(&workspace_bytes, sizeof(workspace_bytes)); put(&st, sizeof(st));
-    const char elev = ctx->allow_elevation ? 1 : 0; put(&elev, 1);
+    const char elev = (ctx->allow_elevation ? 1 : 0) | (ctx->reverse_selection ? 2 : 0); put(&elev, 1);
     for (auto& g : ctx->graphs)
       if (g.key == key) {
         if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return check_cuda(ctx, "backbone_forward (graph launch)");
@@ -685,7 +686,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
       Geometry g = geometry(H, W, lr, pr);
       if ((size_t)g.nW * 8 > 48 * 1024) { result = fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many windows per image (max 6144)"); break; }
       sels[i] = carve_sel(B, H, W, ws.sel + (size_t)i * sel_stride);
-      sargs[i] = make_select_args(sels[i], ws.energy, B, H, W, p->blocks[blk + i].shift, g, 0);
+      sargs[i] = make_select_args(sels[i], ws.energy, B, H, W, p->blocks[blk + i].shift, g, ctx->reverse_selection ? 1 : 0);
     }
     if (result != MIXAQ_OK) break;
     g_launches = 0;
@@ -799,6 +800,12 @@ mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float*
     return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "norm: unsupported C");
   ctx->launches = g_launches;
   return check_cuda(ctx, "norm_forward");
+}
+
+mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  ctx->reverse_selection = reverse != 0;
+  return MIXAQ_OK;
 }
 
 mixaq_status mixaq_set_window_elevation(mixaq_ctx* ctx, int allow) {

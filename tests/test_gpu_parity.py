@@ -230,6 +230,11 @@ def test_precision_classes_within_a_stage_and_the_elevation_switch(orc, mq):
             got = mq.backbone_forward(c, dbb, dev(x), ratios, prunes)[0]
             side.synchronize()
         assert np.array_equal(got.cpu().numpy(), orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=True)[0])
+        # worst-case selection order (Table 4) through the whole backbone
+        c.set_reverse_selection(True)
+        got = mq.backbone_forward(c, dbb, dev(x), ratios, prunes)[0].cpu().numpy()
+        want = orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=True, reverse=True)[0]
+        assert np.array_equal(got, want) and not np.array_equal(got, orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=True)[0])
         assert c.device_status() == 0
     finally:
         c.close()
