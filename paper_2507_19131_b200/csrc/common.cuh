@@ -49,6 +49,50 @@ __device__ __forceinline__ float gelu_f(float v) {
   return __fsub_rn(fmaxf(v, 0.0f), h);
 }
 
+// ---- the same primitives on two values at once (sm_100 packed binary32 arithmetic) --------------------------------
+// __ffma2_rn / __fadd2_rn / __fmul2_rn round each lane like the scalar instruction, so every result below is
+// bit-identical to the scalar function applied to .x and .y; one packed instruction takes one issue slot where two
+// scalar ones take two, which is what the issue-bound epilogues need.  a - b is written fma(b, -1, a): b * -1 is
+// exact, so the single rounding is that of the subtraction.
+__device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, f2(-1.0f), a); }
+
+__device__ __forceinline__ float2 exp2_core2(float2 t) {
+  const float2 r = __fadd2_rn(t, f2(12582912.0f));
+  const float2 nf = __fadd2_rn(r, f2(-12582912.0f));
+  const float2 f = sub2(t, nf);
+  float2 p = f2(__uint_as_float(0x3aafc47du));
+  p = __ffma2_rn(p, f, f2(__uint_as_float(0x3c1e883du)));
+  p = __ffma2_rn(p, f, f2(__uint_as_float(0x3d635716u)));
+  p = __ffma2_rn(p, f, f2(__uint_as_float(0x3e75fc83u)));
+  p = __ffma2_rn(p, f, f2(__uint_as_float(0x3f317219u)));
+  p = __ffma2_rn(p, f, f2(__uint_as_float(0x3f800001u)));
+  return make_float2(__uint_as_float(__float_as_uint(p.x) + (__float_as_uint(r.x) << 23)),
+                     __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(r.y) << 23)));
+}
+
+__device__ __forceinline__ float2 gelu_f2(float2 v) {
+  const float2 a = make_float2(fminf(fabsf(v.x), 5.0f), fminf(fabsf(v.y), 5.0f));
+  float2 q = f2(__uint_as_float(0xb5d6f9e3u));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0x38729e20u)));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0xba6dcc74u)));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0x3c0a3aedu)));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0xbd5c93e3u)));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0xbeeac5d4u)));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0xbf935b8fu)));
+  q = __ffma2_rn(q, a, f2(__uint_as_float(0xbf7fffbeu)));
+  const float2 h = __fmul2_rn(a, exp2_core2(q));
+  return sub2(make_float2(fmaxf(v.x, 0.0f), fmaxf(v.y, 0.0f)), h);
+}
+
+// magic patterns of two values (see quant_magic)
+__device__ __forceinline__ void quant_magic2(float2 x, float inv_scale, float lo, float hi, uint32_t& m0, uint32_t& m1) {
+  float2 t = __fmul2_rn(x, f2(inv_scale));
+  t = make_float2(fminf(fmaxf(t.x, lo), hi), fminf(fmaxf(t.y, lo), hi));
+  t = __fadd2_rn(t, f2(12582912.0f));
+  m0 = __float_as_uint(t.x); m1 = __float_as_uint(t.y);
+}
+
 // q = clamp(rne(x*inv_scale) + zp, 0, qmax), evaluated without a rounding or conversion instruction:
 // rne is monotone and fixes integers, so clamping BEFORE rounding to the integer bounds [-zp, qmax-zp] gives the
 // same code; adding 1.5*2^23 then rounds to nearest-even exactly (|t| <= 255) and leaves 0x4B400000 + rne(t) in

@@ -55,12 +55,14 @@ __device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, b
       const float4 b4 = *reinterpret_cast<const float4*>(cc.bias + lc0 + 4 * i4);
       bb[0] = b4.x; bb[1] = b4.y; bb[2] = b4.z; bb[3] = b4.w;
     }
+    // two columns per packed instruction (each lane rounds like the scalar fma / mul)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < 4; j += 2) {
       const int i = 4 * i4 + j;
-      const float f = __int2float_rn(acc_raw[i] - zz[j]);
-      if (MODE == EPI_MERGE) v[i] = __fmul_rn(f, mm[j]);
-      else                   v[i] = __fmaf_rn(f, mm[j], bb[j]);
+      const float2 f = make_float2(__int2float_rn(acc_raw[i] - zz[j]), __int2float_rn(acc_raw[i + 1] - zz[j + 1]));
+      const float2 r = MODE == EPI_MERGE ? __fmul2_rn(f, make_float2(mm[j], mm[j + 1]))
+                                         : __ffma2_rn(f, make_float2(mm[j], mm[j + 1]), make_float2(bb[j], bb[j + 1]));
+      v[i] = r.x; v[i + 1] = r.y;
     }
   }
 }
@@ -92,8 +94,13 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
       AQ q = br.q0;
       if (MODE == EPI_QKV) { const int sec = n0 / C; if (sec == 1) q = br.q1; else if (sec == 2) q = br.q2; }
       uint32_t c[EPI_NC];
+      const float q_lo = -q.zpf, q_hi = q.qmaxf - q.zpf;
 #pragma unroll
-      for (int i = 0; i < EPI_NC; ++i) c[i] = quant_magic(MODE == EPI_FC1 ? gelu_f(v[i]) : v[i], q);
+      for (int i = 0; i < EPI_NC; i += 2) {
+        float2 g = make_float2(v[i], v[i + 1]);
+        if (MODE == EPI_FC1) g = gelu_f2(g);
+        quant_magic2(g, q.inv_scale, q_lo, q_hi, c[i], c[i + 1]);
+      }
       if (row_ok) {
         uint8_t* dst = out_row + (long)n0 * bits / 8;
         const uint32_t kp = pack_const(q.zp, bits);
