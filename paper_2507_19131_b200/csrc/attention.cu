@@ -174,39 +174,40 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
         const int rqi = sm.rq[i];
         uint32_t xlo = 0, xhi = 0;
         if (SHIFTED) { const uint32_t ri = sm.reg[i] * 0x11111111u; xlo = regj_lo ^ ri; xhi = regj_hi ^ ri; }
-        float lg[7][2];
+        // the two columns a lane holds per key tile are handled as a pair (packed binary32 arithmetic, lane-wise
+        // the same operations as the scalar contract)
+        float2 lg[7];
         float mx = -3.0e38f;
 #pragma unroll
         for (int nt = 0; nt < 7; ++nt) {
           const float4 rb = __ldg(relf + (mt * 7 + nt) * 32);
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int s_int = c[nt][2 * r + u] + rqi + ckj[nt][u];
-            const float rel = r == 0 ? (u == 0 ? rb.x : rb.y) : (u == 0 ? rb.z : rb.w);
-            float v = __fmaf_rn(__int2float_rn(s_int), alpha, rel);
-            if (SHIFTED) {
-              const uint32_t x = nt < 4 ? (xlo >> (4 * (2 * nt + u))) & 15u : (xhi >> (4 * (2 * (nt - 4) + u))) & 15u;
-              v = __fadd_rn(v, x != 0 ? -100.0f : 0.0f);
-            }
-            lg[nt][u] = v;
-            const bool valid = nt < 6 || (t == 0 && u == 0);       // key columns 49..55 do not exist
-            if (valid) mx = fmaxf(mx, v);
+          const float2 sf = make_float2(__int2float_rn(c[nt][2 * r] + rqi + ckj[nt][0]),
+                                        __int2float_rn(c[nt][2 * r + 1] + rqi + ckj[nt][1]));
+          float2 v = __ffma2_rn(sf, f2(alpha), r == 0 ? make_float2(rb.x, rb.y) : make_float2(rb.z, rb.w));
+          if (SHIFTED) {
+            const uint32_t x0 = nt < 4 ? (xlo >> (4 * (2 * nt))) & 15u : (xhi >> (4 * (2 * (nt - 4)))) & 15u;
+            const uint32_t x1 = nt < 4 ? (xlo >> (4 * (2 * nt + 1))) & 15u : (xhi >> (4 * (2 * (nt - 4) + 1))) & 15u;
+            v = __fadd2_rn(v, make_float2(x0 != 0 ? -100.0f : 0.0f, x1 != 0 ? -100.0f : 0.0f));
           }
+          lg[nt] = v;
+          // key columns 49..55 do not exist: of tile 6 only column 0 of lane t = 0
+          if (nt < 6 || t == 0) mx = fmaxf(mx, v.x);
+          if (nt < 6) mx = fmaxf(mx, v.y);
         }
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         // exponentials and this lane's partial sum in column order (the partial of index t of the contract)
         float part = 0.0f;
 #pragma unroll
-        for (int nt = 0; nt < 7; ++nt)
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const bool valid = nt < 6 || (t == 0 && u == 0);
-            float e = exp2_core(fmaxf(__fmul_rn(__fsub_rn(lg[nt][u], mx), kLog2e), -125.0f));
-            e = valid ? e : 0.0f;
-            lg[nt][u] = e;
-            part = __fadd_rn(part, e);
-          }
+        for (int nt = 0; nt < 7; ++nt) {
+          float2 tt = __fmul2_rn(sub2(lg[nt], f2(mx)), f2(kLog2e));
+          tt = make_float2(fmaxf(tt.x, -125.0f), fmaxf(tt.y, -125.0f));
+          float2 e = exp2_core2(tt);
+          if (!(nt < 6 || t == 0)) e.x = 0.0f;
+          if (!(nt < 6)) e.y = 0.0f;
+          lg[nt] = e;
+          part = __fadd_rn(__fadd_rn(part, e.x), e.y);
+        }
         const float s1 = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, 1));
         const float sum = __fadd_rn(s1, __shfl_xor_sync(0xffffffffu, s1, 2));
         const float inv = __fdiv_rn(1.0f, sum);
@@ -214,17 +215,18 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
         int ps = 0;
 #pragma unroll
         for (int nt = 0; nt < 7; ++nt) {
+          float2 tq = __fmul2_rn(__fmul2_rn(lg[nt], f2(inv)), f2(pmaxf));
+          tq = make_float2(fminf(fmaxf(tq.x, 0.0f), pmaxf), fminf(fmaxf(tq.y, 0.0f), pmaxf));
+          tq = __fadd2_rn(tq, f2(12582912.0f));
+          const uint32_t code[2] = {__float_as_uint(tq.x) - kMagicBits, __float_as_uint(tq.y) - kMagicBits};
+          const int ks = nt >> 2, sub = nt & 3;
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
-            float tq = __fmul_rn(__fmul_rn(lg[nt][u], inv), pmaxf);
-            tq = fminf(fmaxf(tq, 0.0f), pmaxf);
-            const uint32_t code = __float_as_uint(__fadd_rn(tq, 12582912.0f)) - kMagicBits;
-            ps += (int)code;
-            const int ks = nt >> 2, sub = nt & 3;
-            pa[ks][r + 2 * (sub >> 1)] |= code << (8 * (2 * (sub & 1) + u));
+            ps += (int)code[u];
+            pa[ks][r + 2 * (sub >> 1)] |= code[u] << (8 * (2 * (sub & 1) + u));
             if (br.tap_p) {
               const int j = 8 * nt + 2 * t + u;
-              if (i < WT && j < WT) br.tap_p[(((long)slot * a.heads + h) * WT + i) * WT + j] = (uint8_t)code;
+              if (i < WT && j < WT) br.tap_p[(((long)slot * a.heads + h) * WT + i) * WT + j] = (uint8_t)code[u];
             }
           }
         }
