@@ -98,21 +98,22 @@ __global__ void __launch_bounds__(256, 4) k_ln_quant_g(LnBranch hi, LnBranch lo,
       for (int k = 0; k < o; ++k) p[k] = __fadd_rn(p[k], p[k + o]);
     return p[0];
   };
+  // neighbouring partials are summed as pairs (packed binary32 arithmetic: each lane adds in the same order)
   float p[P];
 #pragma unroll
-  for (int k = 0; k < P; ++k) {
-    float s = 0.0f;
+  for (int k = 0; k < P; k += 2) {
+    float2 s = f2(0.0f);
 #pragma unroll
-    for (int i = 0; i < NG; ++i) s = __fadd_rn(s, x[i][k]);
-    p[k] = s;
+    for (int i = 0; i < NG; ++i) s = __fadd2_rn(s, make_float2(x[i][k], x[i][k + 1]));
+    p[k] = s.x; p[k + 1] = s.y;
   }
   const float mean = __fdiv_rn(reduce32(p), (float)C);
 #pragma unroll
-  for (int k = 0; k < P; ++k) {
-    float v = 0.0f;
+  for (int k = 0; k < P; k += 2) {
+    float2 v = f2(0.0f);
 #pragma unroll
-    for (int i = 0; i < NG; ++i) { const float d = __fsub_rn(x[i][k], mean); v = __fmaf_rn(d, d, v); }
-    p[k] = v;
+    for (int i = 0; i < NG; ++i) { const float2 d = sub2(make_float2(x[i][k], x[i][k + 1]), f2(mean)); v = __ffma2_rn(d, d, v); }
+    p[k] = v.x; p[k + 1] = v.y;
   }
   const float var = __fdiv_rn(reduce32(p), (float)C);
   const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, 1e-5f)));
@@ -130,11 +131,19 @@ __global__ void __launch_bounds__(256, 4) k_ln_quant_g(LnBranch hi, LnBranch lo,
       const float4 b4 = __ldg(reinterpret_cast<const float4*>(br.beta + 32 * i + P * j) + v4);
       const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
+      for (int e = 0; e < 4; e += 2) {
         const int k = 4 * v4 + e;
-        const uint32_t pat = srow < 0 ? zpat : quant_magic(ln_apply(x[i][k], mean, rstd, gg[e], bb[e]), q);
-        if (k < per) w0 += pat << (bits * k);
-        else         w1 += pat << (bits * (k - per));
+        // y = fma((x - mean) * rstd, gamma, beta) on two channels, then their magic patterns
+        const float2 d = __fmul2_rn(sub2(make_float2(x[i][k], x[i][k + 1]), f2(mean)), f2(rstd));
+        const float2 y = __ffma2_rn(d, make_float2(gg[e], gg[e + 1]), make_float2(bb[e], bb[e + 1]));
+        uint32_t pat[2];
+        quant_magic2(y, q.inv_scale, -q.zpf, q.qmaxf - q.zpf, pat[0], pat[1]);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const uint32_t pt = srow < 0 ? zpat : pat[u];
+          if (k + u < per) w0 += pt << (bits * (k + u));
+          else             w1 += pt << (bits * (k + u - per));
+        }
       }
     }
     // P codes of `bits` bits: P*bits/8 whole bytes (the launcher only picks G with P*bits >= 8)
