@@ -249,15 +249,17 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
       const int i = 16 * mt + g + 8 * r;
 #pragma unroll
       for (int ne = 0; ne < 4; ++ne) {
-        uint32_t two = 0;
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int o_int = d[ne][2 * r + u] - zv * psum[r];
-          if (br.tap_pv && r < nrows && i < WT) br.tap_pv[(m_base + i) * C + h * HEAD_DIM + 8 * ne + 2 * t + u] = o_int;
-          const uint32_t code = quant_code(__fmul_rn(__int2float_rn(o_int), so), oq);
-          two |= code << (8 * u);
+        const int o0 = d[ne][2 * r] - zv * psum[r], o1 = d[ne][2 * r + 1] - zv * psum[r];
+        if (br.tap_pv && r < nrows && i < WT) {
+          int* tp = br.tap_pv + (m_base + i) * C + h * HEAD_DIM + 8 * ne + 2 * t;
+          tp[0] = o0; tp[1] = o1;
         }
-        reinterpret_cast<uint16_t*>(&sm.o[warp][g + 8 * r][0])[4 * ne + t] = (uint16_t)two;
+        // O = O_int * s_p*s_v, then the proj-input quantizer, both columns of the lane at once
+        uint32_t m0, m1;
+        quant_magic2(__fmul2_rn(make_float2(__int2float_rn(o0), __int2float_rn(o1)), f2(so)), oq.inv_scale, -oq.zpf,
+                     oq.qmaxf - oq.zpf, m0, m1);
+        const uint32_t kz = (uint32_t)oq.zp - kMagicBits;
+        reinterpret_cast<uint16_t*>(&sm.o[warp][g + 8 * r][0])[4 * ne + t] = (uint16_t)((m0 + kz) | ((m1 + kz) << 8));
       }
     }
     __syncwarp();
