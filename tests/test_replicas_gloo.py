@@ -41,7 +41,7 @@ def _worker(rank, world, port, out):
 
 def test_two_gloo_ranks_report_the_slowest_time_and_the_whole_job():
     world, port = 2, _free_port()
-    mgr = mp.Manager()
+    mgr = mp.get_context("spawn").Manager()
     out = mgr.dict()
     mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
     for rank in range(world):
