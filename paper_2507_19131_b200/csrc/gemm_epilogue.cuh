@@ -86,13 +86,20 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     // ---- code outputs: every thread quantizes and packs the 16 codes of its own row ----
     if (!acc_ready()) return false;
     const int bits = br.out_bits;
-    uint8_t* out_row = br.out_codes + m * ((long)N * bits / 8);
+    // this thread's output position of the warp's first chunk; packing constants of the (up to three) quantizers
+    uint8_t* out_ptr = br.out_codes + m * ((long)N * bits / 8) + (long)n_first * bits / 8;
+    const int out_step = col_step * bits / 8;
+    const uint32_t kp0 = pack_const(br.q0.zp, bits);
+    const uint32_t kp1 = MODE == EPI_QKV ? pack_const(br.q1.zp, bits) : kp0;
+    const uint32_t kp2 = MODE == EPI_QKV ? pack_const(br.q2.zp, bits) : kp0;
+    const int n_k = C, n_v = 2 * C;                      // first columns of the k and v sections (QKV)
     auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
       const int n0 = n_first + ch * col_step;
       float v[EPI_NC];
       dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
       AQ q = br.q0;
-      if (MODE == EPI_QKV) { const int sec = n0 / C; if (sec == 1) q = br.q1; else if (sec == 2) q = br.q2; }
+      uint32_t kp = kp0;
+      if (MODE == EPI_QKV) { if (n0 >= n_v) { q = br.q2; kp = kp2; } else if (n0 >= n_k) { q = br.q1; kp = kp1; } }
       uint32_t c[EPI_NC];
       const float q_lo = -q.zpf, q_hi = q.qmaxf - q.zpf;
 #pragma unroll
@@ -102,8 +109,7 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
         quant_magic2(g, q.inv_scale, q_lo, q_hi, c[i], c[i + 1]);
       }
       if (row_ok) {
-        uint8_t* dst = out_row + (long)n0 * bits / 8;
-        const uint32_t kp = pack_const(q.zp, bits);
+        uint8_t* dst = out_ptr + ch * out_step;
         if (bits == 8) store_magic<8, EPI_NC>(dst, c, kp);
         else if (bits == 4) store_magic<4, EPI_NC>(dst, c, kp);
         else store_magic<2, EPI_NC>(dst, c, kp);
