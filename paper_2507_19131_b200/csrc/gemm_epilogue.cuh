@@ -137,24 +137,28 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
   const int cj = lane & 3, rsub = lane >> 2;
   long src_mine = -1;
   if (MODE != EPI_MERGE && row_ok) src_mine = br.rowsrc[m];
-  long res_row[4], dst_row[4];            // row offsets (in elements) of the residual and of the output, -1: none
+  // this lane's four (row, 16-byte piece) positions of the warp's first chunk: residual source and output, NULL: none
+  const float* res_ptr[4];
+  float* dst_ptr[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = 8 * i + rsub;
     const long mr = row0 + r;
     const long s = __shfl_sync(0xffffffffu, src_mine, r);
     const bool ok = mr < br.M;
-    if (MODE == EPI_PROJ)     { res_row[i] = (ok && s >= 0) ? s * N : -1;  dst_row[i] = ok ? mr * N : -1; }
-    else if (MODE == EPI_FC2) { res_row[i] = (ok && s >= 0) ? mr * N : -1; dst_row[i] = (ok && s >= 0) ? s * N : -1; }
-    else                      { res_row[i] = -1;                            dst_row[i] = ok ? mr * N : -1; }
+    long res_row, dst_row;               // row offsets (in elements), -1: none
+    if (MODE == EPI_PROJ)     { res_row = (ok && s >= 0) ? s * N : -1;  dst_row = ok ? mr * N : -1; }
+    else if (MODE == EPI_FC2) { res_row = (ok && s >= 0) ? mr * N : -1; dst_row = (ok && s >= 0) ? s * N : -1; }
+    else                      { res_row = -1;                            dst_row = ok ? mr * N : -1; }
+    res_ptr[i] = (MODE != EPI_MERGE && res_row >= 0) ? br.res + res_row + n_first + 4 * cj : nullptr;
+    dst_ptr[i] = dst_row >= 0 ? br.out_f + dst_row + n_first + 4 * cj : nullptr;
   }
   float4 res[4], res_next[4];
   auto fetch = [&](int ch, float4 (&dst)[4]) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);       // a pad token's residual input is zero
-      if (MODE != EPI_MERGE && res_row[i] >= 0)
-        dst[i] = __ldg(reinterpret_cast<const float4*>(br.res + res_row[i] + n_first + ch * col_step + 4 * cj));
+      if (res_ptr[i]) dst[i] = __ldg(reinterpret_cast<const float4*>(res_ptr[i] + ch * col_step));
     }
   };
   if (n_chunks > 0) fetch(0, res);
@@ -174,11 +178,14 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     for (int i = 0; i < 4; ++i) {
       const int r = 8 * i + rsub;
       const float4 a = *reinterpret_cast<const float4*>(stage + r * EPI_NC + 4 * (cj ^ ((r >> 1) & 3)));
-      if (dst_row[i] >= 0) {
-        float4 o;
-        if (MODE == EPI_MERGE) o = a;
-        else o = make_float4(__fadd_rn(res[i].x, a.x), __fadd_rn(res[i].y, a.y), __fadd_rn(res[i].z, a.z), __fadd_rn(res[i].w, a.w));
-        *reinterpret_cast<float4*>(br.out_f + dst_row[i] + n0 + 4 * cj) = o;
+      if (dst_ptr[i]) {
+        float4 o = a;
+        if (MODE != EPI_MERGE) {
+          const float2 lo = __fadd2_rn(make_float2(res[i].x, res[i].y), make_float2(a.x, a.y));
+          const float2 hi = __fadd2_rn(make_float2(res[i].z, res[i].w), make_float2(a.z, a.w));
+          o = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+        *reinterpret_cast<float4*>(dst_ptr[i] + ch * col_step) = o;
       }
     }
     __syncwarp();
