@@ -96,6 +96,14 @@ def lib():
     """Loads libmixaq.so.  Raises if it has not been built: the product has no other code path."""
     global _lib
     if _lib is None:
+        if os.path.abspath(LIB_PATH) == os.path.join(_HERE, "libmixaq.so"):
+            # (re)build when the library is missing or older than its sources; a box without nvcc uses what is there
+            try:
+                from . import build as _build
+                _build.build_library()
+            except Exception as e:                      # noqa: BLE001
+                if not os.path.exists(LIB_PATH):
+                    raise MixaqError(-4, f"{LIB_PATH} is missing and could not be built: {e}")
         if not os.path.exists(LIB_PATH):
             raise MixaqError(-4, f"{LIB_PATH} is missing: build it with paper_2507_19131_b200/build.py")
         L = C.CDLL(LIB_PATH)
