@@ -16,40 +16,7 @@ struct AQ {                   // activation quantizer in kernel-friendly form
   int zp, bits;
 };
 
-__device__ __forceinline__ float magic_round_add() { return 12582912.0f; }   // 1.5 * 2^23
-
-// 2^t by a round-to-nearest split t = n + f and a degree-5 polynomial in f (Horner, fused multiply-adds);
-// n goes straight into the exponent field.  Valid for t in [-125, 127].
-__device__ __forceinline__ float exp2_core(float t) {
-  const float M = 12582912.0f;
-  float r = __fadd_rn(t, M);
-  float nf = __fsub_rn(r, M);
-  float f = __fsub_rn(t, nf);
-  float p = __uint_as_float(0x3aafc47du);
-  p = __fmaf_rn(p, f, __uint_as_float(0x3c1e883du));
-  p = __fmaf_rn(p, f, __uint_as_float(0x3d635716u));
-  p = __fmaf_rn(p, f, __uint_as_float(0x3e75fc83u));
-  p = __fmaf_rn(p, f, __uint_as_float(0x3f317219u));
-  p = __fmaf_rn(p, f, __uint_as_float(0x3f800001u));
-  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(r) << 23));
-}
-
-// GELU(v) = max(v,0) - a*Phi(-a), a = min(|v|, 5); log2 Phi(-a) is a degree-7 polynomial on [0,5].
-__device__ __forceinline__ float gelu_f(float v) {
-  float a = fminf(fabsf(v), 5.0f);
-  float q = __uint_as_float(0xb5d6f9e3u);
-  q = __fmaf_rn(q, a, __uint_as_float(0x38729e20u));
-  q = __fmaf_rn(q, a, __uint_as_float(0xba6dcc74u));
-  q = __fmaf_rn(q, a, __uint_as_float(0x3c0a3aedu));
-  q = __fmaf_rn(q, a, __uint_as_float(0xbd5c93e3u));
-  q = __fmaf_rn(q, a, __uint_as_float(0xbeeac5d4u));
-  q = __fmaf_rn(q, a, __uint_as_float(0xbf935b8fu));
-  q = __fmaf_rn(q, a, __uint_as_float(0xbf7fffbeu));
-  float h = __fmul_rn(a, exp2_core(q));
-  return __fsub_rn(fmaxf(v, 0.0f), h);
-}
-
-// ---- the same primitives on two values at once (sm_100 packed binary32 arithmetic) --------------------------------
+// ---- the floating-point primitives work on two values at once (sm_100 packed binary32 arithmetic) ----------------
 // __ffma2_rn / __fadd2_rn / __fmul2_rn round each lane like the scalar instruction, so every result below is
 // bit-identical to the scalar function applied to .x and .y; one packed instruction takes one issue slot where two
 // scalar ones take two, which is what the issue-bound epilogues need.  a - b is written fma(b, -1, a): b * -1 is
@@ -57,6 +24,8 @@ __device__ __forceinline__ float gelu_f(float v) {
 __device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
 __device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, f2(-1.0f), a); }
 
+// 2^t by a round-to-nearest split t = n + f and a degree-5 polynomial in f (Horner, fused multiply-adds);
+// n goes straight into the exponent field.  Valid for t in [-125, 127].
 __device__ __forceinline__ float2 exp2_core2(float2 t) {
   const float2 r = __fadd2_rn(t, f2(12582912.0f));
   const float2 nf = __fadd2_rn(r, f2(-12582912.0f));
@@ -71,6 +40,7 @@ __device__ __forceinline__ float2 exp2_core2(float2 t) {
                      __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(r.y) << 23)));
 }
 
+// GELU(v) = max(v,0) - a*Phi(-a), a = min(|v|, 5); log2 Phi(-a) is a degree-7 polynomial on [0,5].
 __device__ __forceinline__ float2 gelu_f2(float2 v) {
   const float2 a = make_float2(fminf(fabsf(v.x), 5.0f), fminf(fabsf(v.y), 5.0f));
   float2 q = f2(__uint_as_float(0xb5d6f9e3u));
@@ -210,38 +180,6 @@ __device__ __forceinline__ void store_codes_lane_strided(uint8_t* row, const uin
       uint32_t c3 = __shfl_down_sync(0xffffffffu, c, 3);
       if ((lane & 3) == 0) row[(lane + 32 * i) >> 2] = (uint8_t)(c | (c1 << 2) | (c2 << 4) | (c3 << 6));
     }
-  }
-}
-
-// 32 consecutive codes of one row (held by ONE thread) packed and stored with vector stores.
-// dst points at the first byte of the group; it is 32*bits/8-byte aligned by construction.
-__device__ __forceinline__ void store_codes_32(uint8_t* dst, const uint32_t (&c)[32], int bits) {
-  if (bits == 8) {
-    uint32_t w[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] = c[4 * i] | (c[4 * i + 1] << 8) | (c[4 * i + 2] << 16) | (c[4 * i + 3] << 24);
-    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-    reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-  } else if (bits == 4) {
-    uint32_t w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t v = 0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) v |= c[8 * i + e] << (4 * e);
-      w[i] = v;
-    }
-    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-  } else {
-    uint32_t w[2];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      uint32_t v = 0;
-#pragma unroll
-      for (int e = 0; e < 16; ++e) v |= c[16 * i + e] << (2 * e);
-      w[i] = v;
-    }
-    reinterpret_cast<uint2*>(dst)[0] = make_uint2(w[0], w[1]);
   }
 }
 
