@@ -70,36 +70,44 @@ def sum_range(cost_lo: float, cost_hi: float, n_pairs: int, saving: float = 0.5)
     return ((1.0 - cost_hi) * n_pairs / saving, (1.0 - cost_lo) * n_pairs / saving)
 
 
+def largest_remainder(shares: Sequence[float], total: int, cap: Optional[int] = None) -> np.ndarray:
+    """Apportions `total` indivisible units in proportion to the non-negative `shares` (largest-remainder method):
+    every entry first gets the integer part of its quota; the units still missing go, one each, to the entries with the
+    largest fractional parts.  With `cap`, no entry ends above it: entries at the cap are skipped when the missing
+    units are handed out (needs total <= cap * len(shares))."""
+    shares = np.asarray(shares, dtype=np.float64)
+    if total < 0 or shares.ndim != 1 or shares.size == 0 or (shares < 0).any() or shares.sum() <= 0:
+        raise ValueError("need a non-empty vector of non-negative shares with a positive sum and total >= 0")
+    if cap is not None and total > cap * shares.size:
+        raise ValueError("total cannot be met under the cap")
+    quota = shares * (float(total) / float(shares.sum()))
+    units = np.floor(quota + 1e-12).astype(np.int64)
+    if cap is not None:
+        units = np.minimum(units, cap)
+    while int(units.sum()) < total:
+        open_entries = [i for i in range(shares.size) if cap is None or units[i] < cap]
+        open_entries.sort(key=lambda i: (-(quota[i] - units[i]), i))
+        for i in open_entries[: total - int(units.sum())]:
+            units[i] += 1
+    return units
+
+
 def sample_ratios(rng: np.random.Generator, n: int = 6, s_min: float = 0.6, s_max: float = 4.2, u: float = 0.8,
                   alpha: float = 1.0, max_tries: int = 100000) -> List[float]:
-    """Uniform-sum compression-ratio sampling (Algorithm 1).  Works in tenths: the target sum S is drawn uniformly
-    from the integers of [10 s_min, 10 s_max] (the rounding step needs an integer difference), the split comes from a
-    symmetric Dirichlet (the paper leaves alpha open; 1 = uniform on the simplex), vectors with an entry above the
-    upper bound are rejected, and the largest-remainder method rounds to tenths keeping the sum."""
-    S_lo, S_hi, U = int(round(s_min * 10)), int(round(s_max * 10)), u * 10.0
-    S = int(rng.integers(S_lo, S_hi + 1))
-    if S > n * U + 1e-9:
+    """One ratio vector whose SUM is uniformly distributed (the behaviour of Appendix 6.1, Algorithm 1): ratios are
+    multiples of 0.1, none above `u`, and their sum is uniform over the tenths of [s_min, s_max].
+    The sum is drawn first, as an integer number of tenths; a symmetric Dirichlet draw (the paper leaves its
+    concentration open; alpha = 1 is uniform on the simplex) says how the pairs share it and is redrawn while any
+    pair's share of the sum exceeds the bound; `largest_remainder` turns the shares into whole tenths."""
+    cap = int(round(u * 10))
+    tenths = int(rng.integers(int(np.ceil(s_min * 10 - 1e-9)), int(np.floor(s_max * 10 + 1e-9)) + 1))
+    if tenths > cap * n:
         raise ValueError("target sum cannot be met under the upper bound")
     for _ in range(max_tries):
-        r = rng.dirichlet([alpha] * n) * S
-        if np.all(r <= U + 1e-12):
-            break
-    else:
-        raise RuntimeError("rejection sampling did not terminate")
-    R = np.floor(r + 1e-12).astype(int)
-    diff = S - int(R.sum())
-    if diff > 0:
-        order = np.argsort(-(r - R), kind="stable")
-        for i in range(diff):
-            R[order[i % n]] += 1
-    # an increment can push an entry that sat just under the bound one tenth above it: move the excess on
-    cap = int(round(U))
-    for i in range(n):
-        while R[i] > cap:
-            j = int(np.argmin(R))
-            R[i] -= 1
-            R[j] += 1
-    return [float(v) / 10.0 for v in R]
+        shares = rng.dirichlet(np.full(n, alpha))
+        if shares.max() * tenths <= cap + 1e-12:
+            return [float(k) / 10.0 for k in largest_remainder(shares, tenths, cap)]
+    raise RuntimeError("no admissible split found")
 
 
 def backbone_pair_gmacs(dims: Sequence[int], depths: Sequence[int], H0: int, W0: int, window: int = 7):

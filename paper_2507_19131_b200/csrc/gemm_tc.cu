@@ -13,8 +13,8 @@
 //               the swizzled layout (rows whose byte pitch is no multiple of 16 cannot be described to the TMA
 //               unit and are read with plain loads instead);
 //   then        epilogue (12 warps for the code outputs, 8 for the binary32 outputs): tcgen05.ld (one row per thread, 16 columns per load) + the fused epilogue of the mode.
-// Every wait on an mbarrier is bounded; on expiry the CTA raises the status word, drains, frees its tensor
-// memory and returns.
+// Every wait on an mbarrier is bounded; on expiry the CTA raises the status word, then waits (bounded again) for the
+// copies it has issued to land and for the MMAs it has issued to retire, frees its tensor memory and returns.
 #include <cuda.h>
 #include "gemm_epilogue.cuh"
 
@@ -57,7 +57,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_b
   L.consts_off = L.ring_bytes;                                  // per epilogue warp (zc, mult, bias) x 128 columns
   L.stage_off = L.consts_off + NUM_EPI_WARPS * 3 * EPI_WARP_COLS * 4;   // per epilogue warp 32 x 16 floats
   L.bars_off = L.stage_off + NUM_EPI_WARPS * EPI_STAGE_FLOATS * 4;
-  L.total = L.bars_off + (3 * MAX_RING + 4) * 8 + 16;
+  L.total = L.bars_off + (3 * MAX_RING + 5) * 8 + 16;   // + the drain barrier; then TMEM base, abort flag, fill count
   return L;
 }
 
@@ -144,9 +144,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   float* s_stage = reinterpret_cast<float*>(smem + L.stage_off);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars_off);
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * MAX_RING, bar_raw = bar_empty + 8u * MAX_RING;
-  const uint32_t bar_tfull = bar_raw + 8u * MAX_RING, bar_tempty = bar_tfull + 16u;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 3 * MAX_RING + 4);
+  const uint32_t bar_tfull = bar_raw + 8u * MAX_RING, bar_tempty = bar_tfull + 16u, bar_drain = bar_tempty + 16u;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 3 * MAX_RING + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  volatile int* fills_issued = reinterpret_cast<volatile int*>(tmem_holder + 2);   // k-blocks the TMA thread has issued
+  int my_arrivals = 0;                       // unpack warps: k-blocks this warp has arrived for on the full barriers
 
   constexpr int NUM_EPI_WARPS = epi_warps(MODE);
   constexpr int NUM_UNPACK_WARPS = unpack_warps(MODE), NUM_UNPACK_THREADS = NUM_UNPACK_WARPS * 32;
@@ -173,7 +175,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
       mbar_init(bar_tfull + 8u * a, 1u);                        // tcgen05.commit of the tile's last MMA
       mbar_init(bar_tempty + 8u * a, NUM_EPI_WARPS);            // one arrival per epilogue warp
     }
+    mbar_init(bar_drain, 1u);                                   // tcgen05.commit of the give-up path
     *abort_flag = 0;
+    *fills_issued = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -214,6 +218,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
           }
         }
       }
+      *fills_issued = it;                                       // read by the give-up path only
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -293,6 +298,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
         if (lane == 0) mbar_arrive(bar_full + 8u * s);
       }
     }
+    my_arrivals = it;
     __syncwarp();
   } else {
     // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).. and takes every EPI_SPLIT-th 16-column chunk ----
@@ -344,12 +350,30 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (*abort_flag) {
-    // a wait ran out: report, and give copies already in flight a bounded chance to land before the CTA exits
+    // A wait ran out.  Before the CTA may exit, the copies already issued must have landed in its shared memory and
+    // the MMAs already issued must have retired.  (1) Every unpack warp arrives, on the full barrier of each k-block
+    // that was issued but that it had not reached, so that those phases can complete once their bytes are there
+    // (the ring admits at most one such k-block per stage).  (2) The MMA thread commits what it has issued to a
+    // barrier of its own.  (3) One thread waits, bounded, for the phase of the LAST fill of every stage, on the
+    // packed-rows barrier and on the full barrier, and for the MMA commit.
+    const int issued = *fills_issued;
+    if (warp >= 2 && warp < FIRST_EPI_WARP && lane == 0)
+      for (int j = my_arrivals; j < issued; ++j) mbar_arrive(bar_full + 8u * (uint32_t)(j % p.ring));
+    if (tid == 32) mma_commit(bar_drain);
+    __syncthreads();
     if (tid == 0) {
       atomicExch(p.status, 1);
-      for (int s = 0; s < p.ring; ++s)
-        for (uint32_t it = 0; it < (1u << 16); ++it)
-          if (mbar_try_wait(bar_full + 8u * s, 0) || mbar_try_wait(bar_full + 8u * s, 1)) break;
+      auto drain = [](uint32_t bar, uint32_t parity) {
+        for (uint32_t it = 0; it < (1u << 20); ++it) if (mbar_try_wait(bar, parity)) return;
+      };
+      for (int s = 0; s < p.ring; ++s) {
+        const int fills = issued > s ? (issued - s + p.ring - 1) / p.ring : 0;     // k-blocks j < issued with j % ring == s
+        if (fills == 0) continue;
+        const uint32_t parity = (uint32_t)(fills - 1) & 1u;
+        drain(bar_raw + 8u * s, parity);
+        drain(bar_full + 8u * s, parity);
+      }
+      drain(bar_drain, 0u);
     }
     __syncthreads();
   }

@@ -6,7 +6,9 @@
 
 namespace mixaq {
 
-extern int g_launches;   // kernels launched since the API call started (host bookkeeping)
+// kernels launched since the API call started (host bookkeeping); per thread, so that calls made on different
+// contexts from different threads do not disturb each other's counts
+extern thread_local int g_launches;
 
 // ---- selection ------------------------------------------------------------------------------
 void launch_energy(const float* x, int32_t* energy, long ntok, int C, float inv_scale, cudaStream_t st);

@@ -17,6 +17,7 @@ namespace mixaq {
 bool merge_dim_supported(int C);
 int* ctx_status_word(mixaq_ctx* ctx);
 void ctx_note(mixaq_ctx* ctx, const char* msg, int launches);
+int ctx_device(const mixaq_ctx* ctx);
 }  // namespace mixaq
 
 using namespace mixaq;
@@ -81,6 +82,13 @@ extern "C" mixaq_status mixaq_merge_forward_static(mixaq_ctx* ctx, const mixaq_m
              "use mixaq_merge_forward with a workspace", need, (size_t)MIXAQ_STATIC_SCRATCH_BYTES);
     ctx_note(ctx, msg, 0);
     return MIXAQ_WORKSPACE_TOO_SMALL;
+  }
+  // the array's address is looked up for the CURRENT device: it has to be the one the context was created on
+  int cur_dev = -1;
+  if (cudaGetDevice(&cur_dev) != cudaSuccess || cur_dev != ctx_device(ctx)) {
+    cudaGetLastError();
+    ctx_note(ctx, "merge_forward_static: the current device is not the context's device", 0);
+    return MIXAQ_INVALID_ARG;
   }
   unsigned char* scratch = nullptr;
   cudaError_t e = scratch_address(&scratch);

@@ -13,7 +13,7 @@
 namespace mixaq {
 bool ln_dim_supported(int C);
 bool merge_dim_supported(int C);
-int g_launches = 0;
+thread_local int g_launches = 0;
 }  // namespace mixaq
 
 using namespace mixaq;
@@ -38,6 +38,7 @@ struct mixaq_ctx {
 namespace mixaq {
 // accessors for translation units that do not see the context's layout
 int* ctx_status_word(mixaq_ctx* ctx) { return ctx->d_status; }
+int ctx_device(const mixaq_ctx* ctx) { return ctx->device; }
 void ctx_note(mixaq_ctx* ctx, const char* msg, int launches) {
   if (msg) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
   ctx->launches = launches;
@@ -620,8 +621,8 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "backbone workspace too small");
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
-  // Replay as a CUDA graph when an identical call was captured before.  The key is the exact bytes of everything
-  // that shapes the launches: the HOST parameter structs, ratios, pointers, sizes and the stream.
+  // Replay as a CUDA graph when an identical call was captured before.  The key is made of every value that
+  // shapes the launches: the fields of the HOST parameter structs, ratios, pointers, sizes and the stream.
   bool use_graph = ctx->graph_cache && !ctx->profiling && st != nullptr && st != cudaStreamLegacy;
   if (use_graph) {
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
@@ -629,11 +630,34 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   }
   std::string key;
   if (use_graph) {
+    // field by field: the structs contain padding bytes whose content the caller does not control
     auto put = [&key](const void* ptr, size_t n) { key.append((const char*)ptr, n); };
+    auto put_aq = [&](const mixaq_aq& q) { put(&q.bits, 4); put(&q.scale, 4); put(&q.inv_scale, 4); put(&q.zero_point, 4); };
+    auto put_lin = [&](const mixaq_linear& l) {
+      put(&l.codes, sizeof(l.codes)); put(&l.scale, sizeof(l.scale)); put(&l.out_features, 4); put(&l.in_features, 4); put(&l.bits, 4);
+    };
+    auto put_branch = [&](const mixaq_branch& b) {
+      const float* ptrs[8] = {b.ln1_g, b.ln1_b, b.ln2_g, b.ln2_b, b.b_qkv, b.b_proj, b.b_fc1, b.b_fc2};
+      put(ptrs, sizeof(ptrs));
+      put_aq(b.qkv_in); put_aq(b.q); put_aq(b.k); put_aq(b.v); put_aq(b.proj_in); put_aq(b.fc1_in); put_aq(b.fc2_in);
+      put(&b.bits, 4);
+    };
     const int npairs = (nblk + 1) / 2;
     put(&p->num_stages, sizeof(int)); put(p->depths, sizeof(int) * p->num_stages);
-    put(p->blocks, sizeof(mixaq_block_params) * nblk);
-    if (p->num_stages > 1) put(p->merges, sizeof(mixaq_merge_params) * (p->num_stages - 1));
+    for (int b = 0; b < nblk; ++b) {
+      const mixaq_block_params& q = p->blocks[b];
+      const int dims[5] = {q.dim, q.heads, q.window, q.shift, q.hidden};
+      put(dims, sizeof(dims));
+      put_lin(q.qkv); put_lin(q.proj); put_lin(q.fc1); put_lin(q.fc2);
+      put(&q.relpos_table, sizeof(q.relpos_table));
+      put_branch(q.hi); put_branch(q.lo);
+      put(&q.score_inv_scale, 4); put(&q.prepared, sizeof(q.prepared));
+    }
+    for (int m = 0; m + 1 < p->num_stages; ++m) {
+      const mixaq_merge_params& q = p->merges[m];
+      put(&q.ln_g, sizeof(q.ln_g)); put(&q.ln_b, sizeof(q.ln_b)); put_aq(q.in); put_lin(q.reduction);
+      put(&q.prepared, sizeof(q.prepared));
+    }
     put(&x0, sizeof(x0)); put(stage_out, sizeof(float*) * p->num_stages);
     const int dims[3] = {B, H0, W0}; put(dims, sizeof(dims));
     put(low_ratio_per_pair, sizeof(float) * npairs);

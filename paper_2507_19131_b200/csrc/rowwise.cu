@@ -215,7 +215,6 @@ void launch_ln_npl(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
   else if (RMAX >= 2 && rows >= 2 * 8 * 148 * 4) launch_ln_r<NPL, (RMAX >= 2 ? 2 : RMAX)>(hi, lo, st);
   else launch_ln_r<NPL, 1>(hi, lo, st);
 }
-#define MIXAQ_NPL_CASE(n, KERNEL, ...) case n: KERNEL<n><<<grid, 256, 0, st>>>(__VA_ARGS__); break;
 #define MIXAQ_LN_CASE(n, rmax) case n: launch_ln_npl<n, rmax>(hi, lo, st); break;
 
 template <int NG, int G>

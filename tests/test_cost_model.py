@@ -92,6 +92,17 @@ def test_largest_remainder_rounding_keeps_the_sum():
         assert round(sum(r) * 10) == 20
 
 
+def test_largest_remainder_apportionment_closed_forms():
+    lr = cm.largest_remainder
+    assert lr([1, 1, 1], 10).tolist() == [4, 3, 3]                 # equal remainders: lowest index first
+    assert lr([0.5, 0.3, 0.2], 10).tolist() == [5, 3, 2]           # exact quotas
+    assert lr([0.47, 0.33, 0.20], 7).tolist() == [3, 2, 2]         # quotas 3.29, 2.31, 1.40: the 0.40 remainder wins
+    assert lr([0.9, 0.05, 0.05], 10, cap=8).tolist() == [8, 1, 1]  # the capped entry's excess moves on
+    assert lr([3, 1], 0).tolist() == [0, 0]
+    with pytest.raises(ValueError):
+        lr([1, 1], 17, cap=8)
+
+
 def test_real_shape_macs_are_in_the_papers_range():
     """The paper's 14.16 GMACs per stage-3 pair is the linear-layer cost of 4000 tokens; our 800x1333 shape has
     50x84 = 4200 tokens padded to 56x84."""
