@@ -99,6 +99,7 @@ typedef struct {
  * branch's bit width; accumulators are zero-point corrected int32. */
 typedef struct {
   uint8_t* a_codes;   int32_t* qkv_acc;  uint8_t* qkv_codes;
+  float*   probs;     /* [slots][heads][49][49], the binary32 softmax output before its quantizer */
   uint8_t* p_codes;   /* [slots][heads][49][49], one code per byte */
   int32_t* pv_acc;    uint8_t* o_codes;  int32_t* proj_acc;  float* x1;
   uint8_t* f1_codes;  int32_t* fc1_acc;  uint8_t* f2_codes;  int32_t* fc2_acc;

@@ -490,9 +490,108 @@ void orc_block_forward(const orc_block* p, const float* x, float* y, int B, int 
   }
 }
 
+// The uniform quantized Swin block, written on the WHOLE map in the published order of a Swin block (norm -> zero
+// padding -> cyclic shift -> window partition -> attention -> reverse -> crop -> FFN) and token by token in global
+// coordinates.  It shares only the scalar primitives above (quantizer, LayerNorm row, softmax row, GELU, dequantize)
+// with the two-branch path: no window gathering, no per-window mask or bias table, no batch bookkeeping.  Ratio 0 and
+// ratio 1 of orc_block_forward must reproduce it bit for bit (Section 3.3: the ratio is the share of low windows).
+static void uniform_block_quant_whole_map(const orc_block& P, const orc_branch& br, const float* x, float* y,
+                                          int B, int H, int W) {
+  const int C = P.dim, ws = P.window, nh = P.heads, d = C / nh, Hd = P.hidden, s = P.shift;
+  const int Hp = round_up(H, ws), Wp = round_up(W, ws);
+  const long NP = (long)Hp * Wp;
+  const int pmax = (1 << br.bits) - 1;
+  const orc_aq pq = { br.bits, 1.0f / (float)pmax, (float)pmax, 0 };
+  const float alpha = (br.q.scale * br.k.scale) * (float)(1.0 / std::sqrt((double)d));
+  const float so = pq.scale * br.v.scale;
+  auto region = [&](int pos, int L) { return pos < L - ws ? 0 : (pos < L - s ? 1 : 2); };
+  for (int b = 0; b < B; ++b) {
+    const float* xb = x + (long)b * H * W * C;
+    float* yb = y + (long)b * H * W * C;
+    // 1. LayerNorm of the real tokens, zero padding AFTER the norm, input quantizer, QKV projection, q/k/v quantizers
+    std::vector<uint8_t> qkv(NP * 3 * C);
+#pragma omp parallel for schedule(static)
+    for (long tok = 0; tok < NP; ++tok) {
+      const int ty = (int)(tok / Wp), tx = (int)(tok % Wp);
+      std::vector<float> ln(C, 0.0f);
+      if (ty < H && tx < W) layernorm_row(xb + ((long)ty * W + tx) * C, C, br.ln1_g, br.ln1_b, ln.data());
+      std::vector<uint8_t> a(C);
+      for (int c = 0; c < C; ++c) a[c] = quant1(ln[c], br.qkv_in);
+      for (int n = 0; n < 3 * C; ++n) {
+        int32_t acc = 0;
+        for (int c = 0; c < C; ++c) acc += ((int)a[c] - br.qkv_in.zp) * (int)P.qkv.codes[(long)n * C + c];
+        const float v = dequant_bias(acc, br.qkv_in.scale, P.qkv.scale[n], br.b_qkv[n]);
+        qkv[tok * 3 * C + n] = quant1(v, n < C ? br.q : (n < 2 * C ? br.k : br.v));
+      }
+    }
+    // 2. every real token attends the tokens of its window in the cyclically shifted frame (pad tokens are keys),
+    //    then proj + residual, LN2, fc1, GELU, fc2 + residual
+#pragma omp parallel for schedule(dynamic, 16)
+    for (long tok = 0; tok < NP; ++tok) {
+      const int ty = (int)(tok / Wp), tx = (int)(tok % Wp);
+      if (ty >= H || tx >= W) continue;                       // cropped away at the end
+      const int ys = (ty - s + Hp) % Hp, xs = (tx - s + Wp) % Wp;       // my position in the shifted frame
+      const int wy0 = ys / ws * ws, wx0 = xs / ws * ws;                 // my window's corner in the shifted frame
+      const int iy = ys - wy0, ix = xs - wx0;
+      const int my_reg = region(ys, Hp) * 3 + region(xs, Wp);
+      const int T = ws * ws;
+      std::vector<long> key(T);
+      std::vector<int> key_reg(T);
+      for (int j = 0; j < T; ++j) {
+        const int ky = wy0 + j / ws, kx = wx0 + j % ws;
+        key[j] = (long)((ky + s) % Hp) * Wp + (kx + s) % Wp;
+        key_reg[j] = region(ky, Hp) * 3 + region(kx, Wp);
+      }
+      std::vector<float> logits(T), prob(T);
+      std::vector<uint8_t> pc(T), o(C);
+      for (int h = 0; h < nh; ++h) {
+        for (int j = 0; j < T; ++j) {
+          int32_t sdot = 0;
+          for (int e = 0; e < d; ++e)
+            sdot += ((int)qkv[tok * 3 * C + h * d + e] - br.q.zp) * ((int)qkv[key[j] * 3 * C + C + h * d + e] - br.k.zp);
+          const int ridx = (iy - j / ws + ws - 1) * (2 * ws - 1) + (ix - j % ws + ws - 1);
+          float lg = std::fmaf((float)sdot, alpha, P.relpos[(long)ridx * nh + h]);
+          if (s > 0) lg = lg + (key_reg[j] == my_reg ? 0.0f : -100.0f);
+          logits[j] = lg;
+        }
+        softmax_row(logits.data(), T, prob.data());
+        for (int j = 0; j < T; ++j) pc[j] = quant1(prob[j], pq);
+        for (int e = 0; e < d; ++e) {
+          int32_t pv = 0;
+          for (int j = 0; j < T; ++j) pv += (int)pc[j] * ((int)qkv[key[j] * 3 * C + 2 * C + h * d + e] - br.v.zp);
+          o[h * d + e] = quant1((float)pv * so, br.proj_in);
+        }
+      }
+      const float* xr = xb + ((long)ty * W + tx) * C;
+      std::vector<float> x1(C), ln(C);
+      for (int n = 0; n < C; ++n) {
+        int32_t acc = 0;
+        for (int c = 0; c < C; ++c) acc += ((int)o[c] - br.proj_in.zp) * (int)P.proj.codes[(long)n * C + c];
+        x1[n] = xr[n] + dequant_bias(acc, br.proj_in.scale, P.proj.scale[n], br.b_proj[n]);
+      }
+      layernorm_row(x1.data(), C, br.ln2_g, br.ln2_b, ln.data());
+      std::vector<uint8_t> f1(C), f2(Hd);
+      for (int c = 0; c < C; ++c) f1[c] = quant1(ln[c], br.fc1_in);
+      for (int n = 0; n < Hd; ++n) {
+        int32_t acc = 0;
+        for (int c = 0; c < C; ++c) acc += ((int)f1[c] - br.fc1_in.zp) * (int)P.fc1.codes[(long)n * C + c];
+        f2[n] = quant1(gelu1(dequant_bias(acc, br.fc1_in.scale, P.fc1.scale[n], br.b_fc1[n])), br.fc2_in);
+      }
+      float* yr = yb + ((long)ty * W + tx) * C;
+      for (int n = 0; n < C; ++n) {
+        int32_t acc = 0;
+        for (int c = 0; c < Hd; ++c) acc += ((int)f2[c] - br.fc2_in.zp) * (int)P.fc2.codes[(long)n * Hd + c];
+        yr[n] = x1[n] + dequant_bias(acc, br.fc2_in.scale, P.fc2.scale[n], br.b_fc2[n]);
+      }
+    }
+  }
+}
+
 void orc_uniform_block_forward(const orc_block* p, const orc_branch* br, const float* x, float* y,
                                int B, int H, int W) {
   const orc_block& P = *p;
+  if (P.quant) { uniform_block_quant_whole_map(P, *br, x, y, B, H, W); return; }
+  // fp mode (all quantizers off; pinned to a textbook Swin block in binary64): window by window
   const int ws = P.window, T = ws * ws;
   const int Hp = round_up(H, ws), Wp = round_up(W, ws), nW = (Hp / ws) * (Wp / ws);
   std::vector<float> relb((long)P.heads * T * T);

@@ -105,7 +105,9 @@ void  orc_block_forward(const orc_block* p, const float* x, float* y, int B, int
                         double low_ratio, double prune_ratio, const int32_t* energy, int reverse,
                         int32_t* order_out, uint8_t* cls_out, int64_t* score_out,
                         const orc_taps* taps_hi, const orc_taps* taps_lo);
-/* a uniform quantized Swin block: every window in natural order through ONE branch; no selection code */
+/* a uniform quantized Swin block through ONE branch, written separately on the whole map, token by token in global
+ * coordinates (norm -> pad -> shift -> partition); shares only the scalar primitives with orc_block_forward.
+ * (With quant = 0 it runs the fp-mode windows in natural order.) */
 void  orc_uniform_block_forward(const orc_block* p, const orc_branch* br, const float* x, float* y,
                                 int B, int H, int W);
 void  orc_merge_forward(const orc_merge* m, const float* x, int B, int H, int W, int C, float* y);

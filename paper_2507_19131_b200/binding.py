@@ -75,7 +75,7 @@ class Selection(C.Structure):
     _fields_ = [("cls", C.c_void_p), ("order", C.c_void_p), ("score", C.c_void_p)]
 
 
-_TAP_FIELDS = ("a_codes", "qkv_acc", "qkv_codes", "p_codes", "pv_acc", "o_codes", "proj_acc", "x1",
+_TAP_FIELDS = ("a_codes", "qkv_acc", "qkv_codes", "probs", "p_codes", "pv_acc", "o_codes", "proj_acc", "x1",
                "f1_codes", "fc1_acc", "f2_codes", "fc2_acc")
 
 
@@ -293,7 +293,7 @@ def _alloc_taps(device, M, slots, Cc, hidden, heads, bits):
     z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
     t = SimpleNamespace(
         a_codes=z((M, Cc * bits // 8), u8), qkv_acc=z((M, 3 * Cc), i32), qkv_codes=z((M, 3 * Cc * bits // 8), u8),
-        p_codes=z((slots, heads, 49, 49), u8), pv_acc=z((M, Cc), i32), o_codes=z((M, Cc * bits // 8), u8),
+        probs=z((slots, heads, 49, 49), f32), p_codes=z((slots, heads, 49, 49), u8), pv_acc=z((M, Cc), i32), o_codes=z((M, Cc * bits // 8), u8),
         proj_acc=z((M, Cc), i32), x1=z((M, Cc), f32), f1_codes=z((M, Cc * bits // 8), u8),
         fc1_acc=z((M, hidden), i32), f2_codes=z((M, hidden * bits // 8), u8), fc2_acc=z((M, Cc), i32))
     s = BranchTaps()

@@ -215,7 +215,14 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
         int ps = 0;
 #pragma unroll
         for (int nt = 0; nt < 7; ++nt) {
-          float2 tq = __fmul2_rn(__fmul2_rn(lg[nt], f2(inv)), f2(pmaxf));
+          const float2 pr = __fmul2_rn(lg[nt], f2(inv));          // the softmax output itself
+          if (br.tap_probs) {
+            const int j0 = 8 * nt + 2 * t;
+            float* tp = br.tap_probs + (((long)slot * a.heads + h) * WT + i) * WT;
+            if (i < WT && j0 < WT) tp[j0] = pr.x;
+            if (i < WT && j0 + 1 < WT) tp[j0 + 1] = pr.y;
+          }
+          float2 tq = __fmul2_rn(pr, f2(pmaxf));
           tq = make_float2(fminf(fmaxf(tq.x, 0.0f), pmaxf), fminf(fmaxf(tq.y, 0.0f), pmaxf));
           tq = __fadd2_rn(tq, f2(12582912.0f));
           const uint32_t code[2] = {__float_as_uint(tq.x) - kMagicBits, __float_as_uint(tq.y) - kMagicBits};

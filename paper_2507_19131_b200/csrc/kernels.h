@@ -93,6 +93,7 @@ struct AttnBranch {
   float alpha;               // s_q*s_k/sqrt(d)
   float so;                  // s_p*s_v
   uint8_t* tap_p;            // nullable
+  float* tap_probs;          // nullable: softmax output [slots][heads][49][49]
   int32_t* tap_pv;           // nullable
 };
 struct AttnArgs {

@@ -455,7 +455,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     ab.bits = brp[i]->bits; ab.slots = slots[i];
     ab.alpha = (brp[i]->q.scale * brp[i]->k.scale) * rs;
     ab.so = (1.0f / (float)((1 << brp[i]->bits) - 1)) * brp[i]->v.scale;
-    ab.tap_p = tp[i] ? tp[i]->p_codes : nullptr; ab.tap_pv = tp[i] ? tp[i]->pv_acc : nullptr;
+    ab.tap_p = tp[i] ? tp[i]->p_codes : nullptr; ab.tap_probs = tp[i] ? tp[i]->probs : nullptr; ab.tap_pv = tp[i] ? tp[i]->pv_acc : nullptr;
   }
   { PROF(PC_ATTN); launch_attention(aa, st); }
 

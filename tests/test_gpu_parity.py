@@ -50,6 +50,8 @@ def check_taps(orc, blk, ref, got, counts):
             assert np.array_equal(g.__dict__[f].cpu().numpy(), orc.pack(r.__dict__[f], bits)), f"{name}.{f}"
         for f in ("qkv_acc", "pv_acc", "proj_acc", "fc1_acc", "fc2_acc", "p_codes"):
             assert np.array_equal(g.__dict__[f].cpu().numpy(), r.__dict__[f]), f"{name}.{f}"
+        assert_close_rel(g.probs.cpu().numpy(), r.probs)                     # the binary32 softmax, stated tolerance
+        assert np.array_equal(g.probs.cpu().numpy(), r.probs), f"{name}.probs not bit-identical"
         assert_close_rel(g.x1.cpu().numpy(), r.x1)
         assert np.array_equal(g.x1.cpu().numpy(), r.x1), f"{name}.x1 not bit-identical"
 
@@ -272,9 +274,10 @@ def _full_backbone_case(orc, mq, ctx, wl):
     torch.cuda.current_stream().wait_stream(side)
 
 
-def test_config3_swin_t_800x1333_full_size(orc, mq, ctx):
-    """Swin-T, 200x334 tokens, W4, A8/A4, ratio 0.25: the benchmark workload."""
-    _full_backbone_case(orc, mq, ctx, synth.config3(ratio=0.25))
+@pytest.mark.parametrize("ratio", [0.0, 0.25, 0.5, 0.75])
+def test_config3_swin_t_800x1333_full_size(orc, mq, ctx, ratio):
+    """Swin-T, 200x334 tokens, W4, A8/A4: the benchmark workload at every low-bit ratio the benchmark sweeps."""
+    _full_backbone_case(orc, mq, ctx, synth.config3(ratio=ratio))
 
 
 def test_config4_swin_s_1024_full_size_three_classes(orc, mq, ctx):

@@ -170,9 +170,9 @@ def test_fp_mode_equals_textbook_swin_block(orc, H, W, shift, dim, heads):
 # ------------------------------------------------------------------------------------------------
 # quantized block internals against numpy restatements built from the taps
 # ------------------------------------------------------------------------------------------------
-def test_quantized_attention_brute_force_from_codes(orc):
+@pytest.mark.parametrize("H,W", [(14, 21), (10, 12)])      # 10 x 12 is padded to 14 x 14: pad tokens are keys
+def test_quantized_attention_brute_force_from_codes(orc, H, W):
     blk = small_block(seed=12, dim=64, heads=2, shift=3)
-    H, W = 14, 21
     x = small_input(10, 1, H, W, 64)
     r = orc.block_forward(blk, x, 0.5, taps=True)
     T, C, nh, d = 49, 64, 2, 32
@@ -208,24 +208,47 @@ def test_quantized_attention_brute_force_from_codes(orc):
         assert near_tie <= 3
 
 
-def test_quantized_block_taps_against_primitives_in_numpy(orc):
+def numpy_window_map(H, W, ws, shift):
+    """[nW][ws*ws] source token (y*W + x) of every window position, -1 for a pad token, from numpy.roll on the padded
+    index map: pad to multiples of the window, roll by -shift, cut into windows."""
+    Hp, Wp = -(-H // ws) * ws, -(-W // ws) * ws
+    idx = -np.ones((Hp, Wp), np.int64)
+    idx[:H, :W] = np.arange(H * W).reshape(H, W)
+    idx = np.roll(idx, (-shift, -shift), axis=(0, 1))
+    return idx.reshape(Hp // ws, ws, Wp // ws, ws).transpose(0, 2, 1, 3).reshape(-1, ws * ws)
+
+
+@pytest.mark.parametrize("H,W,shift", [(14, 14, 0), (10, 12, 3), (16, 19, 3)])
+def test_quantized_block_taps_against_primitives_in_numpy(orc, H, W, shift):
     """Every stage of one quantized window batch restated with numpy from the previous tap: pins the
-    wiring (which quantizer, which bias, which residual) rather than the primitives."""
-    blk = small_block(seed=13, dim=32, heads=1, shift=0, share_bias=False)
-    x = small_input(11, 1, 14, 14, 32)
+    wiring (which quantizer, which bias, which residual) rather than the primitives.  On the ragged, shifted maps the
+    windows hold pad tokens: their rows must carry the code of zero after LN1 (not the norm of a zero row), take part
+    in the layers like any row (residual input zero) and never reach the output map."""
+    blk = small_block(seed=13, dim=32, heads=1, shift=shift, share_bias=False)
+    x = small_input(11, 1, H, W, 32)
     r = orc.block_forward(blk, x, 0.5, taps=True)
     T, C = 49, 32
+    wmap = numpy_window_map(H, W, 7, shift)
+    xf = x[0].reshape(H * W, C)
+    covered = np.zeros(H * W, int)
+    n_pad_rows = 0
     for name, br, off, n in (("hi", blk.hi, 0, r.counts[0]), ("lo", blk.lo, r.counts[0], r.counts[1])):
         tp = getattr(r, name)
         for j in range(n):
             w = int(r.order[0, off + j])
-            wy, wx = divmod(w, 2)
-            xin = x[0, wy * 7:wy * 7 + 7, wx * 7:wx * 7 + 7].reshape(T, C)
+            src = wmap[w]
+            real = src >= 0
+            n_pad_rows += int((~real).sum())
+            xin = np.zeros((T, C), F32)
+            xin[real] = xf[src[real]]
             rows = slice(j * T, (j + 1) * T)
-            a = orc.quantize(orc.layernorm(xin, br.ln1_g, br.ln1_b), br.qkv_in)
+            a = np.empty((T, C), np.uint8)
+            a[real] = orc.quantize(orc.layernorm(xin[real], br.ln1_g, br.ln1_b), br.qkv_in)
+            a[~real] = br.qkv_in.zp                                   # zero AFTER the norm: code of 0.0 is the zero point
             assert np.array_equal(tp.a_codes[rows], a)
             acc = (a.astype(np.int64) - br.qkv_in.zp) @ blk.qkv.codes.astype(np.int64).T
             assert np.array_equal(tp.qkv_acc[rows], acc)
+            assert not acc[~real].any()                               # a pad row enters QKV as exact zeros: q, k, v = bias
             yq = (acc.astype(F32) * (F32(br.qkv_in.scale) * blk.qkv.scale)[None]).astype(np.float64) + br.b_qkv
             for i, qz in enumerate((br.q, br.k, br.v)):
                 want = np.clip(np.rint(yq[:, i * C:(i + 1) * C] * np.float64(F32(qz.inv_scale))) + qz.zp, 0, (1 << qz.bits) - 1)
@@ -249,8 +272,29 @@ def test_quantized_block_taps_against_primitives_in_numpy(orc):
             a2 = (tp.f2_codes[rows].astype(np.int64) - br.fc2_in.zp) @ blk.fc2.codes.astype(np.int64).T
             assert np.array_equal(tp.fc2_acc[rows], a2)
             yw = tp.x1[rows] + a2 * (np.float64(F32(br.fc2_in.scale)) * blk.fc2.scale.astype(np.float64))[None] + br.b_fc2
-            got = r.y[0, wy * 7:wy * 7 + 7, wx * 7:wx * 7 + 7].reshape(T, C)
-            assert np.abs(got - yw).max() < 1e-5 * max(1, np.abs(yw).max())
+            got = r.y[0].reshape(H * W, C)[src[real]]                 # only real tokens are written back
+            assert np.abs(got - yw[real]).max() < 1e-5 * max(1, np.abs(yw).max())
+            covered[src[real]] += 1
+    assert (covered == 1).all()                                        # every token of the map comes from exactly one window row
+    Hp, Wp = -(-H // 7) * 7, -(-W // 7) * 7
+    assert n_pad_rows == Hp * Wp - H * W
+
+
+def test_uniform_block_is_written_separately_and_catches_a_planted_pad_mistake(orc):
+    """The whole-map uniform block and the window-batch path agree bit for bit on a ragged, shifted map (that is the
+    ratio-0 / ratio-1 pin); a plausible mistake -- treating pad tokens as zeros BEFORE the norm, i.e. giving them the
+    code of beta instead of the code of zero -- is visible in the taps the agreement rests on."""
+    blk = small_block(seed=17, dim=32, heads=1, shift=3)
+    x = small_input(18, 1, 10, 12, 32)
+    r = orc.block_forward(blk, x, 0.0, taps=True)
+    assert np.array_equal(r.y, orc.uniform_block_forward(blk, "hi", x))
+    wmap = numpy_window_map(10, 12, 7, 3)
+    zero_code = blk.hi.qkv_in.zp
+    beta_code = orc.quantize(orc.layernorm(np.zeros((1, 32), F32), blk.hi.ln1_g, blk.hi.ln1_b), blk.hi.qkv_in)[0]
+    assert (beta_code != zero_code).any()                              # the two readings differ on this block
+    for j in range(r.counts[0]):
+        pad = wmap[int(r.order[0, j])] < 0
+        assert (r.hi.a_codes[j * 49:(j + 1) * 49][pad] == zero_code).all()
 
 
 def test_sqnr_rises_with_bit_width(orc):

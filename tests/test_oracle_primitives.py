@@ -123,6 +123,24 @@ def test_gelu_vs_erf_form_float64(orc):
     assert abs(x[i] + 0.7518) < 2e-3 and abs(got[i] - want.min()) < 3e-6 and abs(want.min() + 0.16997) < 1e-5
 
 
+def test_contract_polynomials_are_the_minimax_fits_the_fit_script_derives(orc):
+    """The frozen coefficient words of 2^f and log2 Phi(-a) against a fresh Remez run (oracle/fit_contract_polynomials):
+    same polynomial up to the last bits of the small coefficients, maximum error within a few percent of the optimum;
+    and the oracle evaluates exactly those words (Horner, fused multiply-adds) -- checked through orc.exp2 / orc.gelu."""
+    from oracle import fit_contract_polynomials as fit
+    res = fit.check()
+    assert res["exp2"]["max_rel_coef_diff"] < 2e-6 and res["log2_phi_neg"]["max_rel_coef_diff"] < 2e-4
+    for r in res.values():
+        assert r["max_err_frozen"] < 1.08 * r["max_err_fitted"]
+    # the oracle's exp2 on [-1/2, 1/2] is the frozen polynomial evaluated in binary32
+    f = np.linspace(-0.5, 0.5, 1001).astype(F32)
+    c = [F32(fit.word_to_float(w)) for w in fit.FROZEN["exp2"]]
+    p = np.full_like(f, c[5])
+    for k in range(4, -1, -1):
+        p = (p.astype(np.float64) * f.astype(np.float64) + np.float64(c[k])).astype(F32)     # one rounding: a fused multiply-add
+    assert np.array_equal(orc.exp2(f), p)
+
+
 def test_softmax_rows(orc):
     rng = np.random.default_rng(11)
     s = (rng.standard_normal((200, 49)) * 4).astype(F32)
