@@ -28,7 +28,8 @@ if ROOT not in sys.path:
 
 METRIC = "swin_t_two_branch_backbone_images_per_sec_800x1333"
 UNIT = "images/s"
-SWEEP = [0.0, 0.25, 0.5, 0.75]
+SWEEP = [0.0, 0.25, 0.5, 0.75]                     # config 3 (the metric's axis)
+SWEEP_BY_CONFIG = {3: SWEEP, 4: [0.0, 0.25, 0.5, 0.75], 5: [round(0.1 * i, 1) for i in range(9)]}   # config 5: 0 ... 0.8
 L2_FLUSH_BYTES = 256 << 20
 
 
@@ -150,17 +151,26 @@ def algorithmic_work(wl, mq):
 
 
 # The fc1 epilogue (zero-point correction, dequantize, GELU, quantize, pack) is a fixed sequence of binary32 / integer
-# lane operations per output, set by the numeric contract: 3 (int subtract, convert, fma) + 20 (GELU: |v| clamp, 7 fma,
-# 3 adds of the rounding split, 5 fma, exponent insert, multiply, max, subtract) + 4 (quantize) + 1 (pack) = 28.
-# With K = C <= 768 the MMA needs K/64 <= 12 clocks per output row-chunk where the epilogue needs 28 issue slots, so
-# the kernel is bound by plain ALU issue; its peak is SMs x 128 lanes x SM clock.
+# lane operations per output, set by the numeric contract (28 scalar operations); with K = C <= 768 the MMA needs
+# K/64 <= 12 clocks per output row-chunk, so this family is bound by instruction issue, not by the tensor pipe.
 FC1_EPILOGUE_OPS = 28
-ALU_CATS = {"gemm_fc1_gelu"}
-NUM_SMS, LANES_PER_SM = 148, 128
+NUM_SMS = 148
 TENSOR_CATS = {"gemm_qkv", "gemm_proj", "gemm_fc1_gelu", "gemm_fc2_scatter", "gemm_merge"}
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None
-# (stage-1 launch of the category, the largest of its 12 launches per step; profiles/gemm_tc_stage1_ncu_full.md)
-NCU_TRAFFIC_PER_LAUNCH = {"gemm_fc1_gelu": 5.03e6, "gemm_fc2_scatter": 47.1e6, "gemm_qkv": 5.01e6, "gemm_proj": 31.1e6}
+
+
+def recorded_traffic(workload_name):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture) per kernel family of this
+    workload, from profiles/ncu_dram_traffic.json; None when there is no record for the workload or the kernels have
+    changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+    try:
+        rec = json.load(open(path)).get(workload_name)
+    except Exception:
+        return None
+    from paper_2507_19131_b200.ncu_summary import kernel_source_digest
+    if not rec or rec.get("kernel_source_digest") != kernel_source_digest():
+        return None
+    return rec
 
 
 def run_ours(args):
@@ -268,7 +278,26 @@ def run_ours(args):
         comp.wait_stream(s_out); comp.wait_stream(s_in)
         t_end.record(comp)
         barrier()
-        return dict(ms=replicas.max_over_ranks(t_begin.elapsed_time(t_end), device="cuda"), wl=wl, h2d=x_host.numel() * 4, d2h=sum(h.numel() * 4 for h in sets[0]["host"]))
+        ms = replicas.max_over_ranks(t_begin.elapsed_time(t_end), device="cuda")
+        h2d, d2h = x_host.numel() * 4, sum(h.numel() * 4 for h in sets[0]["host"])
+
+        # what the host link gives these very buffers, each direction alone (the pipeline cannot be faster than the
+        # slower of the two): 5 copies each, CUDA events on the copying stream
+        def link_gbs(stream, fn, nbytes, reps=5):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                fn()
+                a.record(stream)
+                for _ in range(reps):
+                    fn()
+                b_.record(stream)
+            stream.synchronize()
+            return nbytes * reps / (a.elapsed_time(b_) * 1e-3) / 1e9
+        b0 = sets[0]
+        up = link_gbs(s_in, lambda: b0["x"].copy_(x_host, non_blocking=True), h2d)
+        down = link_gbs(s_out, lambda: [h.copy_(o, non_blocking=True) for h, o in zip(b0["host"], b0["dbb"].outs)], d2h)
+        barrier()
+        return dict(ms=ms, wl=wl, h2d=h2d, d2h=d2h, h2d_gbs=up, d2h_gbs=down)
 
     sampler = ClockSampler(local) if rank == 0 else None
     main = time_ratio(args.ratio, K, Wm, sampler)
@@ -293,29 +322,53 @@ def run_ours(args):
     tot = sum(v["ms_per_step"] for v in kernels.values()) or 1.0
     for v in kernels.values():
         v["share"] = round(v["ms_per_step"] / tot, 4)
+    # Roofline: the path's contractions are the five GEMM families; their aggregate rate (useful int8 operations of one
+    # forward over the summed CUDA-event time of the GEMM launches) against the int8 tensor peak = 2 x the measured bf16
+    # peak (nominal int8 : bf16 ratio).  Each launch is bracketed by its own events, i.e. timed alone: the burst figure
+    # is the denominator; the fraction against the sustained figure is given beside it.
+    gemm_cats = [c for c in kernels if c in TENSOR_CATS]
+    gemm_ms = sum(kernels[c]["ms_per_step"] for c in gemm_cats)
+    gemm_ops = sum(work[c]["ops"] for c in gemm_cats)
+    gemm_launches = sum(kernels[c]["launches_per_step"] for c in gemm_cats)
+    peak_burst, peak_sust = 2.0 * peaks["bf16_burst"], 2.0 * peaks["bf16_sustained"]
+    agg_tops = gemm_ops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    rec = recorded_traffic(main["wl"].name)
+    traffic = None
+    if rec:
+        try:
+            traffic = sum(rec["bytes_per_step"][c] for c in gemm_cats) / max(1, gemm_launches)
+        except Exception:
+            traffic = None
     dom = max(kernels, key=lambda c: kernels[c]["ms_per_step"])
-    dk = kernels[dom]
-    if dom in ALU_CATS:
-        clk = (main["clocks"] or {}).get("sm_mhz") or 1965.0
-        peak = NUM_SMS * LANES_PER_SM * clk * 1e6 / 1e12          # T lane-ops/s at the SM clock sampled under load
-        ach = work[dom]["alu_ops"] / (dk["ms_per_step"] * 1e-3) / 1e12
-        roof = dict(kernel=dom, bound="alu", achieved=round(ach, 3), peak=round(peak, 3), unit="T lane-op/s",
-                    frac=round(ach / peak, 5),
-                    peak_source="148 SMs x 128 lanes x sampled SM clock; 28 contract operations per fc1 output",
-                    tensor_tops=dk["tops"], tensor_frac=round(dk["tops"] / (2.0 * peaks["bf16_sustained"]), 5))
-    elif dom in TENSOR_CATS:
-        peak = 2.0 * peaks["bf16_sustained"]      # int8 dense = 2 x bf16 (nominal ratio) on the measured bf16 peak
-        roof = dict(kernel=dom, bound="tensor", achieved=dk["tops"], peak=peak, unit="TOP/s(int8)",
-                    frac=round(dk["tops"] / peak, 5),
-                    peak_source=f"2 x bf16_tflops_sustained of {peaks['source']} peaks (kernel timed inside a long step)")
-    else:
-        peak = peaks["hbm_gbs"]
-        roof = dict(kernel=dom, bound="hbm", achieved=dk["gbs"], peak=peak, unit="GB/s",
-                    frac=round(dk["gbs"] / peak, 5), peak_source=f"hbm_gbs of {peaks['source']} peaks")
-    roof["launch_us"] = round(1e3 * dk["ms_per_step"] / max(1, dk["launches_per_step"]), 3)
-    roof["traffic"] = NCU_TRAFFIC_PER_LAUNCH.get(dom)
-    roof["traffic_note"] = "dram bytes of the category's stage-1 launch (ncu); activations are largely L2-resident"
-    roof["timed"] = "separate pass of K steps with CUDA events around every kernel, on the launching stream"
+    clk = (main["clocks"] or {}).get("sm_mhz") or 1965.0
+    roof = dict(kernel="k_gemm_tc (QKV, proj, fc1+GELU, fc2+scatter, merge: all GEMM launches of one forward)",
+                bound="tensor", achieved=round(agg_tops, 3), peak=round(peak_burst, 1), unit="TOP/s(int8)",
+                frac=round(agg_tops / peak_burst, 5), frac_of_sustained=round(agg_tops / peak_sust, 5),
+                peak_source=f"2 x bf16_tflops (burst) of {peaks['source']} peaks; sustained: 2 x bf16_tflops_sustained",
+                launches_per_step=gemm_launches, launch_us=round(1e3 * gemm_ms / max(1, gemm_launches), 3),
+                gemm_ms_per_step=round(gemm_ms, 5), gemm_gop_per_step=round(gemm_ops / 1e9, 2),
+                traffic=traffic,
+                traffic_note=("mean dram bytes per GEMM launch (ncu, profiles/ncu_dram_traffic.json)" if traffic is not None else
+                              "no ncu record for these kernel sources and this workload"),
+                per_family={c: dict(tops=kernels[c]["tops"], tensor_frac_burst=round(kernels[c]["tops"] / peak_burst, 5),
+                                    tensor_frac_sustained=round(kernels[c]["tops"] / peak_sust, 5),
+                                    ms_per_step=kernels[c]["ms_per_step"]) for c in gemm_cats},
+                dominant_kernel=dom,
+                timed="separate pass of K steps with CUDA events around every kernel, on the launching stream")
+    if "gemm_fc1_gelu" in kernels:
+        # what bounds the code-output epilogues: instruction issue.  Warp instructions per output come from the ncu
+        # counter smsp__inst_executed of the recorded capture when there is one.
+        fk = kernels["gemm_fc1_gelu"]
+        outs = work["gemm_fc1_gelu"]["alu_ops"] / FC1_EPILOGUE_OPS
+        issue_peak = NUM_SMS * 4 * clk * 1e6                    # warp instructions per second: 4 schedulers per SM
+        note = dict(kernel="gemm_fc1_gelu", outputs_per_step=int(outs),
+                    outputs_per_s=round(outs / (fk["ms_per_step"] * 1e-3) / 1e12, 4), unit="T outputs/s")
+        wi = (rec or {}).get("fc1_warp_inst_per_32_outputs")
+        if wi:
+            note.update(warp_inst_per_32_outputs=wi,
+                        issue_frac=round(outs / 32.0 * wi / (fk["ms_per_step"] * 1e-3) / issue_peak, 4),
+                        issue_peak="148 SMs x 4 schedulers x sampled SM clock; instruction count from ncu smsp__inst_executed")
+        roof["alu_note"] = note
 
     # end to end through the public call with HOST buffers (pinned): every step copies its image host->device, runs
     # the forward and copies the four stage maps device->host.  Two buffer sets and three streams let the copies of
@@ -325,7 +378,7 @@ def run_ours(args):
 
     sweep = {}
     if args.sweep and world == 1:
-        for r in SWEEP:
+        for r in SWEEP_BY_CONFIG[CONFIG]:
             if abs(r - args.ratio) < 1e-9:
                 sweep[str(r)] = round(value, 2)
                 continue
@@ -337,43 +390,44 @@ def run_ours(args):
     bbm = main["wl"].backbone
     pair_g, fixed_g = cm.backbone_pair_gmacs(bbm.dims, bbm.depths, main["wl"].H, main["wl"].W)
     cost = {str(r): {"relative_bops": round(cm.relative_cost([r] * len(pair_g), pair_g, fixed_g), 4),
-                     "equivalent_act_bits": round(cm.equivalent_act_bits([r] * len(pair_g), 8.0, pair_g, fixed_g), 3)}
-            for r in (SWEEP if args.sweep else [args.ratio])}
+                     "equivalent_act_bits": round(cm.equivalent_act_bits([r] * len(pair_g), float(bbm.blocks[0].hi.bits), pair_g, fixed_g), 3)}
+            for r in (SWEEP_BY_CONFIG[CONFIG] if args.sweep else [args.ratio])}
 
-    # the steps on either side of the path (patch embedding of the raw image, LayerNorm of the four stage maps)
+    # the same forward with the steps on either side of the path inside the call and its graph: raw image ->
+    # patch embedding -> two-branch backbone -> LayerNorm of the four stage maps (one mixaq_backbone_forward call)
     stem = None
     if CONFIG == 3 and world == 1:
         from paper_2507_19131_b200 import synth
         rng = np.random.default_rng(77)
+        wl_s = main["wl"]
         emb = synth.make_embed(rng, bbm.dims[0])
-        de = mq.DeviceEmbed(ctx, emb)
-        img = torch.from_numpy(synth.input_image(78, main["wl"].B, 800, 1333)).cuda()
-        gb = [(torch.ones(c, device="cuda"), torch.zeros(c, device="cuda")) for c in bbm.dims]
-        outs = main["dbb"].outs
-        x0 = mq.embed_forward(ctx, de, img)
-
-        def timed(fn, n=20):
-            for _ in range(3):
-                fn()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(n):
-                fn()
-            b.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) * 1e3 / n
-        stem = {"patch_embed_us": round(timed(lambda: mq.embed_forward(ctx, de, img, x0)), 2),
-                "stage_norms_us": round(timed(lambda: [mq.norm_forward(ctx, g, b, o, o) for (g, b), o in zip(gb, outs)]), 2),
-                "note": "800x1333x3 image -> 200x334x96 tokens (3 launches); LayerNorm of the 4 stage maps (4 launches); "
-                        "stream launches, not part of `value`"}
+        norms = [(np.ones(c, np.float32), np.zeros(c, np.float32)) for c in bbm.dims]
+        dbs = mq.DeviceBackbone(ctx, wl_s.backbone, wl_s.B, 800, 1333, embed=emb, norms=norms)
+        img = torch.from_numpy(synth.input_image(78, wl_s.B, 800, 1333)).cuda()
+        for _ in range(3):
+            mq.backbone_forward(ctx, dbs, img, wl_s.low_ratios, wl_s.prune_ratios)
+        n_s = max(5, K)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_s)]
+        for i in range(n_s):
+            flush.fill_(i & 0xFF)
+            evs[i][0].record()
+            mq.backbone_forward(ctx, dbs, img, wl_s.low_ratios, wl_s.prune_ratios)
+            evs[i][1].record()
+        torch.cuda.synchronize()
+        ms_s = sum(a.elapsed_time(b) for a, b in evs) / n_s
+        stem = {"value": round(wl_s.B / (ms_s * 1e-3), 2), "unit": UNIT, "ms_per_step": round(ms_s, 4),
+                "launches_per_step": ctx.launch_count(),
+                "note": "800x1333x3 image -> patch embedding -> backbone -> LayerNorm of the 4 stage maps, one call, one graph"}
 
     # tensor-core issue rate as the library's own MMA loop reaches it (context for the tensor fractions above)
     mma_peak = None
     if world == 1:
         mma_peak = {"kind_i8_tops": round(ctx.measure_mma_peak(0, 8000), 1),
                     "kind_f8f6f4_e4m3_tops": round(ctx.measure_mma_peak(1, 8000), 1),
-                    "note": "all SMs issue 128x256x32 tcgen05.mma from shared memory into TMEM; f8f6f4 is the path that "
-                            "carries 4/6-bit operand formats: it is not faster than i8, so no narrower MMA path is used"}
+                    "kind_mxf4_e2m1_tops": round(ctx.measure_mma_peak(2, 8000), 1),
+                    "note": "all SMs issue 128x256xK tcgen05.mma from shared memory into TMEM (K = 32; mxf4: K = 64 from the "
+                            "same bytes).  f8f6f4 carries the 4/6-bit formats in 8-bit containers and is not faster than i8; "
+                            "mxf4 is the block-scaled E2M1 path (grid 0, 1/2, 1, 3/2, 2, 3, 4, 6 and their negatives)"}
 
     status = ctx.device_status()
     if rank != 0:
@@ -386,7 +440,7 @@ def run_ours(args):
         "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int8 MMA (int32 accumulate) + f32 epilogues", "data": "synthetic",
         "config": {"workload": main["wl"].name,
-                   "model": "two-branch Swin backbone, dims %s depths %s" % (bbm.dims, bbm.depths),
+                   "dims": list(bbm.dims), "depths": list(bbm.depths),
                    "tokens": [main["wl"].H, main["wl"].W], "batch_per_gpu": main["wl"].B,
                    "weights": "W%d (int8 container)" % bbm.blocks[0].qkv.bits,
                    "act_bits_high_low": [bbm.blocks[0].hi.bits, bbm.blocks[0].lo.bits], "low_ratio": args.ratio,
@@ -396,13 +450,17 @@ def run_ours(args):
         "clocks": main["clocks"],
         "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
                 "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": round(e2e["ms"] / K, 4),
-                "pipeline": "2 buffer sets, copy-in / compute / copy-out streams; K steps timed as one pipeline"},
+                "pipeline": "2 buffer sets, copy-in / compute / copy-out streams; K steps timed as one pipeline",
+                "host_link_gbs": {"h2d": round(e2e["h2d_gbs"], 2), "d2h": round(e2e["d2h_gbs"], 2)},
+                "link_bound_ms_per_step": round(max(e2e["h2d"] / e2e["h2d_gbs"], e2e["d2h"] / e2e["d2h_gbs"]) / 1e6, 4),
+                "note": "the four binary32 stage maps leave the device every step; when link_bound_ms_per_step exceeds "
+                        "ms_per_step of the resident run, the end-to-end figure is set by this host's PCIe link, not by the kernels"},
         "gpu_launches": main["launches"] * K,
         "roofline": roof,
         "kernels": kernels,
         "low_ratio_sweep_images_per_sec": sweep,
         "paper_cost_model": cost,
-        "stem_and_norms": stem,
+        "value_with_stem": stem,
         "mma_issue_rate": mma_peak,
         "device_status": status,
     }
@@ -529,12 +587,14 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=[3, 4, 5],
                     help="3: Swin-T 800x1333 B=1 (the metric's workload); 4: Swin-S 1024^2 B=4 A4/A2 + 20 %% pruned; 5: Swin-B 1536^2 B=2")
     ap.add_argument("--no-sweep", dest="sweep", action="store_false")
+    ap.add_argument("--sweep", dest="force_sweep", action="store_true",
+                    help="also sweep the low-bit ratio for --config 4 (0 ... 0.75) or 5 (0 ... 0.8); config 3 sweeps by default")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     args = ap.parse_args()
     global CONFIG
     CONFIG = args.config
     if CONFIG != 3:
-        args.sweep = False
+        args.sweep = bool(args.force_sweep)
     if args.impl == "reference":
         run_reference(args)
     else:

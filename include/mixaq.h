@@ -92,6 +92,8 @@ typedef struct {
   uint8_t* cls;            /* [B][nW]  0 high, 1 low, 2 pruned                                              */
   int32_t* order;          /* [B][nW]  window index by rank: first n_hi high, next n_lo low, last n_pr pruned */
   int64_t* score;          /* [B][nW]  window scores                                                         */
+  int32_t *idx_hi, *idx_lo, *idx_pr;   /* [B][n_hi], [B][n_lo], [B][n_pr]: the windows of each class per image, in
+                                          ascending window index (the counts are those of mixaq_branch_counts)   */
 } mixaq_selection;
 
 /* Optional debug taps of one branch (each pointer may be NULL).  Rows are in window-batch order: window slot
@@ -111,6 +113,14 @@ typedef struct {
   const int* depths;                    /* HOST array [num_stages]; every depth is even or 1                */
   const mixaq_block_params* blocks;     /* HOST array, sum(depths) entries                                  */
   const mixaq_merge_params* merges;     /* HOST array, num_stages-1 entries                                 */
+  /* Optional steps on either side of the path (Appendix 6.2 counts them among the layers whose cost is not reduced).
+   * embed != NULL: the `x0` argument of mixaq_backbone_forward is the IMAGE [B][H0][W0][3] and the patch embedding
+   * runs first (the token map is ceil(H0/4) x ceil(W0/4)).  out_norm_g / out_norm_b != NULL (HOST arrays of
+   * num_stages device pointers, both or neither): stage_out[s] receives LayerNorm(stage map s) with these parameters,
+   * while the un-normalised map (kept in the workspace) feeds the next stage. */
+  const mixaq_embed_params* embed;
+  const float* const* out_norm_g;
+  const float* const* out_norm_b;
 } mixaq_backbone_params;
 
 /* ---- context ---- */
@@ -198,8 +208,9 @@ mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float*
 
 /* ---- the backbone: for every stage [merge] -> stage energy -> blocks; one ratio per pair of consecutive
  *      blocks (Section 3.3), optional prune ratio per pair (Section 3.4).  x0 is the [B][H0][W0][C0] map after the
- *      patch-embedding stem; stage_out is a HOST array of num_stages device pointers receiving each stage's final
- *      map [B][Hs][Ws][Cs].  Ratio arrays are HOST arrays with one entry per block pair. ---- */
+ *      patch-embedding stem (or, when p->embed is set, the [B][H0][W0][3] image itself); stage_out is a HOST array of
+ *      num_stages device pointers receiving each stage's final map [B][Hs][Ws][Cs] (normalised when p->out_norm_* are
+ *      set).  Ratio arrays are HOST arrays with one entry per block pair. ---- */
 size_t       mixaq_backbone_workspace_bytes(const mixaq_backbone_params* p, int B, int H0, int W0);
 mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params* p, const float* x0,
                                     float* const* stage_out, int B, int H0, int W0,
@@ -229,12 +240,16 @@ mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse);
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 
-/* ---- tensor-core issue rate as this library reaches it (the denominator for the GEMMs' tensor-pipe fraction):
- *      all SMs at once issue `groups` x 4 tcgen05.mma of 128 x 256 x 32 from shared-memory operands into TMEM.
- *      kind 0: kind::i8 (u8 x s8 -> s32), the path the GEMMs use.  kind 1: kind::f8f6f4 with E4M3 operands, the path
- *      that also carries the 4-bit and 6-bit operand formats (in 8-bit containers): its rate bounds what a narrower
- *      operand type could give.  `scratch`: >= 8 KiB of device memory.  Synchronises the stream; result in 10^12
- *      operations (2 per multiply-accumulate) per second. ---- */
+/* ---- tensor-core issue rate as this library reaches it (the denominator for the GEMMs' tensor-pipe fraction, and the
+ *      measurement behind the choice of MMA kind for the low-bit branch):
+ *      all SMs at once issue `groups` x 4 tcgen05.mma of 128 x 256 x K from shared-memory operands into TMEM.
+ *      kind 0: kind::i8 (u8 x s8 -> s32, K = 32), the path the GEMMs use.
+ *      kind 1: kind::f8f6f4 with E4M3 operands (K = 32), the path that also carries the 4-bit and 6-bit operand formats
+ *              in 8-bit containers: its rate bounds what those formats could give.
+ *      kind 2: kind::mxf4, block-scaled E2M1 operands packed two per byte (K = 64, one UE8M0 scale per 32 values; the
+ *              scale factors are left uninitialised, so the products mean nothing -- only the rate is measured).
+ *      `scratch`: >= 8 KiB of device memory.  Synchronises the stream; result in 10^12 operations (2 per
+ *      multiply-accumulate) per second. ---- */
 mixaq_status mixaq_measure_mma_peak(mixaq_ctx* ctx, int kind, int groups, void* scratch, size_t scratch_bytes,
                                     double* tera_ops_per_s, void* cuda_stream);
 
@@ -247,6 +262,10 @@ int          mixaq_profile_categories(void);
 const char*  mixaq_profile_category_name(int category);
 mixaq_status mixaq_profile_begin(mixaq_ctx* ctx);
 mixaq_status mixaq_profile_end(mixaq_ctx* ctx, void* cuda_stream, float* ms_per_category, int* launches_per_category);
+/* The same, launch by launch in issue order: fills category[i] and ms[i] for the first `capacity` bracketed launches
+ * since mixaq_profile_begin and stores their total number in *count (which may exceed capacity).  Ends the profiling
+ * like mixaq_profile_end. */
+mixaq_status mixaq_profile_end_records(mixaq_ctx* ctx, void* cuda_stream, int* category, float* ms, int capacity, int* count);
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,7 @@ EXPORTS = [
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
-    "mixaq_norm_forward", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
+    "mixaq_norm_forward", "mixaq_profile_end_records", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -72,7 +72,8 @@ class SelectOpts(C.Structure):
 
 
 class Selection(C.Structure):
-    _fields_ = [("cls", C.c_void_p), ("order", C.c_void_p), ("score", C.c_void_p)]
+    _fields_ = [("cls", C.c_void_p), ("order", C.c_void_p), ("score", C.c_void_p),
+                ("idx_hi", C.c_void_p), ("idx_lo", C.c_void_p), ("idx_pr", C.c_void_p)]
 
 
 _TAP_FIELDS = ("a_codes", "qkv_acc", "qkv_codes", "probs", "p_codes", "pv_acc", "o_codes", "proj_acc", "x1",
@@ -89,7 +90,8 @@ class Taps(C.Structure):
 
 class BackboneS(C.Structure):
     _fields_ = [("num_stages", C.c_int), ("depths", C.POINTER(C.c_int)), ("blocks", C.POINTER(BlockS)),
-                ("merges", C.POINTER(MergeS))]
+                ("merges", C.POINTER(MergeS)), ("embed", C.POINTER(EmbedS)),
+                ("out_norm_g", C.POINTER(C.c_void_p)), ("out_norm_b", C.POINTER(C.c_void_p))]
 
 
 def lib():
@@ -174,7 +176,7 @@ class Context:
         self.check(lib().mixaq_selftest_wait_timeout(self.h, _stream_ptr()), "selftest_wait_timeout")
 
     def measure_mma_peak(self, kind: int = 0, groups: int = 2000) -> float:
-        """Tensor-core issue rate in TOP/s (kind 0: kind::i8; 1: kind::f8f6f4 with E4M3 operands)."""
+        """Tensor-core issue rate in TOP/s (kind 0: kind::i8; 1: kind::f8f6f4 with E4M3 operands; 2: kind::mxf4)."""
         scratch = torch.empty(8192, dtype=torch.uint8, device=self.device)
         out = C.c_double()
         self.check(lib().mixaq_measure_mma_peak(self.h, kind, groups, _ptr(scratch), C.c_size_t(8192), C.byref(out),
@@ -193,6 +195,13 @@ class Context:
         ms, cnt = (C.c_float * n)(), (C.c_int * n)()
         self.check(lib().mixaq_profile_end(self.h, _stream_ptr(), ms, cnt), "profile_end")
         return {lib().mixaq_profile_category_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
+
+    def profile_end_records(self, capacity: int = 4096):
+        """Returns [(category name, milliseconds)] launch by launch, in issue order, since profile_begin."""
+        cat, ms, n = (C.c_int * capacity)(), (C.c_float * capacity)(), C.c_int()
+        self.check(lib().mixaq_profile_end_records(self.h, _stream_ptr(), cat, ms, capacity, C.byref(n)), "profile_end_records")
+        names = [lib().mixaq_profile_category_name(i).decode() for i in range(lib().mixaq_profile_categories())]
+        return [(names[cat[i]], float(ms[i])) for i in range(min(n.value, capacity))]
 
     def close(self):
         if self.h:
@@ -320,7 +329,9 @@ def block_forward(ctx: Context, db: DeviceBlock, x: torch.Tensor, low_ratio: flo
         out.cls = torch.empty((B, nW), dtype=torch.uint8, device=x.device)
         out.order = torch.empty((B, nW), dtype=torch.int32, device=x.device)
         out.scores = torch.empty((B, nW), dtype=torch.int64, device=x.device)
-        sel = Selection(_ptr(out.cls), _ptr(out.order), _ptr(out.scores))
+        n_hi, n_lo, n_pr = out.counts
+        out.idx_hi, out.idx_lo, out.idx_pr = (torch.empty((B, n), dtype=torch.int32, device=x.device) for n in (n_hi, n_lo, n_pr))
+        sel = Selection(_ptr(out.cls), _ptr(out.order), _ptr(out.scores), _ptr(out.idx_hi), _ptr(out.idx_lo), _ptr(out.idx_pr))
     tp = None
     if taps:
         n_hi, n_lo, _ = out.counts
@@ -408,16 +419,27 @@ def merge_forward_static(ctx: Context, dm: DeviceMerge, x: torch.Tensor, y: torc
 
 
 class DeviceBackbone:
-    """All parameters of a backbone on the device, prepared; owns the workspace and the stage outputs."""
+    """All parameters of a backbone on the device, prepared; owns the workspace and the stage outputs.
+    embed: stem parameters (object with ln_g, ln_b, bias, aq, proj) -- the forward then takes the IMAGE [B,H0,W0,3];
+    norms: one (gamma, beta) pair of numpy vectors per stage -- the stage outputs are then LayerNormed."""
 
-    def __init__(self, ctx: Context, bb, B: int, H0: int, W0: int):
+    def __init__(self, ctx: Context, bb, B: int, H0: int, W0: int, embed=None, norms=None):
         self.ctx, self.bb, self.B, self.H0, self.W0 = ctx, bb, B, H0, W0
         self.dev = _Dev(ctx.device)
         nb = len(bb.blocks)
         self.blocks = (BlockS * nb)(*[fill_block_struct(self.dev, b) for b in bb.blocks])
         self.merges = (MergeS * max(1, len(bb.merges)))(*[fill_merge_struct(self.dev, m) for m in bb.merges])
         self.depths = (C.c_int * len(bb.depths))(*bb.depths)
-        self.s = BackboneS(len(bb.depths), self.depths, self.blocks, self.merges)
+        self.s = BackboneS(len(bb.depths), self.depths, self.blocks, self.merges, None, None, None)
+        self.embed = None
+        if embed is not None:
+            self.embed = DeviceEmbed(ctx, embed)
+            self.s.embed = C.pointer(self.embed.s)
+        if norms is not None:
+            ns = len(bb.depths)
+            self.norm_g = (C.c_void_p * ns)(*[self.dev.up(g, np.float32) for g, _ in norms])
+            self.norm_b = (C.c_void_p * ns)(*[self.dev.up(b, np.float32) for _, b in norms])
+            self.s.out_norm_g, self.s.out_norm_b = self.norm_g, self.norm_b
         for i in range(nb):
             ctx.check(lib().mixaq_block_prepare(ctx.h, C.byref(self.blocks[i]), _stream_ptr()), "block_prepare")
         for i in range(len(bb.merges)):
@@ -426,7 +448,8 @@ class DeviceBackbone:
         if need == 0:
             raise MixaqError(-1, "backbone_workspace_bytes returned 0")
         self.ws = torch.empty(need, dtype=torch.uint8, device=ctx.device)
-        self.outs, h, w = [], H0, W0
+        h, w = ((H0 + 3) // 4, (W0 + 3) // 4) if embed is not None else (H0, W0)
+        self.outs = []
         for s, c in enumerate(bb.dims):
             if s > 0:
                 h, w = (h + 1) // 2, (w + 1) // 2

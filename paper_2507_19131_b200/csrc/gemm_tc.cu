@@ -511,8 +511,11 @@ void launch_wait_probe(int* status, cudaStream_t st) {
 // then waits (bounded) for the commit.  KIND 0: kind::i8 (u8 x s8 -> s32), the path the GEMMs use.
 // KIND 1: kind::f8f6f4 with E4M3 operands (-> f32); this is also the path that carries 4-bit and 6-bit operand
 // formats on sm_100a (in 8-bit shared-memory containers), so its rate bounds what a narrower operand type could give.
+// KIND 2: kind::mxf4 (E2M1 operands packed two per byte, one UE8M0 scale per 32 values, -> f32): 128 x 256 x 64 per
+// instruction from the same 32 bytes per row, the only narrower path with a higher nominal rate.
 template <int KIND>
 __global__ void __launch_bounds__(128, 1) k_mma_peak(int groups, unsigned long long* ns_out, int* status) {
+  constexpr uint32_t PEAK_TMEM_COLS = KIND == 2 ? 512u : 256u;   // KIND 2 keeps its scale factors behind the accumulator
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -525,7 +528,7 @@ __global__ void __launch_bounds__(128, 1) k_mma_peak(int groups, unsigned long l
   if (tid == 0) { mbar_init(smem_u32(bar), 1u); asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(256u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(PEAK_TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -534,8 +537,13 @@ __global__ void __launch_bounds__(128, 1) k_mma_peak(int groups, unsigned long l
   const uint32_t tmem_base = *tmem_holder;
   if (tid == 0) {
     // instruction descriptor: D format (s32 = 2 / f32 = 1) at bit 4, A format at 7, B format at 10, N/8 at 17, M/16 at 24
+    // (block-scaled kinds: no D format field; A and B format 1 = E2M1 at bits 7 and 10, scale format 1 = UE8M0 at bit 23)
     const uint32_t idesc = KIND == 0 ? ((2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(MAX_BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24))
-                                     : ((1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(MAX_BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24));
+                         : KIND == 1 ? ((1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(MAX_BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24))
+                                     : ((1u << 7) | (1u << 10) | ((uint32_t)(MAX_BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24));
+    // KIND 2: the scale factors of A and B sit in tensor memory behind the accumulator (columns 256.., 264..); their
+    // contents are whatever the allocation holds -- the products are meaningless, only the issue rate is measured
+    const uint32_t sfa = tmem_base + 256u, sfb = tmem_base + 264u;
     const uint64_t adesc = smem_desc_sw128(base), bdesc = smem_desc_sw128(base + A_STAGE_BYTES);
     unsigned long long t0, t1;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
@@ -544,6 +552,14 @@ __global__ void __launch_bounds__(128, 1) k_mma_peak(int groups, unsigned long l
         const uint32_t accumulate = (g > 0 || kk > 0) ? 1u : 0u;
         if (KIND == 0) {
           mma_i8(tmem_base, adesc + (uint64_t)(kk * (UMMA_K >> 4)), bdesc + (uint64_t)(kk * (UMMA_K >> 4)), idesc, accumulate);
+        } else if (KIND == 2) {
+          // 32 bytes of a row are 64 E2M1 values: one MMA of 128 x 256 x 64 with one UE8M0 scale per 32 values
+          asm volatile(
+              "{\n\t.reg .pred p;\n\t"
+              "setp.ne.b32 p, %4, 0;\n\t"
+              "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+              ::"r"(tmem_base), "l"(adesc + (uint64_t)(kk * (UMMA_K >> 4))), "l"(bdesc + (uint64_t)(kk * (UMMA_K >> 4))),
+                "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb) : "memory");
         } else {
           asm volatile(
               "{\n\t.reg .pred p;\n\t"
@@ -562,7 +578,7 @@ __global__ void __launch_bounds__(128, 1) k_mma_peak(int groups, unsigned long l
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(PEAK_TMEM_COLS) : "memory");
 }
 
 // ns_out: one entry per SM (device memory).  Returns the grid size, 0 on failure.
@@ -572,9 +588,12 @@ int launch_mma_peak(int kind, int groups, unsigned long long* ns_out, int* statu
   if (kind == 0) {
     if (cudaFuncSetAttribute(k_mma_peak<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
     k_mma_peak<0><<<sms, 128, smem, st>>>(groups, ns_out, status);
-  } else {
+  } else if (kind == 1) {
     if (cudaFuncSetAttribute(k_mma_peak<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
     k_mma_peak<1><<<sms, 128, smem, st>>>(groups, ns_out, status);
+  } else {
+    if (cudaFuncSetAttribute(k_mma_peak<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+    k_mma_peak<2><<<sms, 128, smem, st>>>(groups, ns_out, status);
   }
   ++g_launches;
   return sms;

@@ -27,6 +27,8 @@ struct SelectArgs {
 };
 // selections of `count` blocks that share one energy map (all blocks of a stage): 2 launches per 24 blocks
 void launch_select(const SelectArgs* a, int count, cudaStream_t st);
+// ascending window indices of one class per image: out[b][0 .. n_c) from cls[b][0 .. nW); c = 0, 1, 2 in one launch
+void launch_class_lists(const uint8_t* cls, int B, int nW, int32_t* const out[3], const int count[3], cudaStream_t st);
 
 // ---- row-wise LayerNorm + quantize + pack -----------------------------------------------------
 struct LnBranch {

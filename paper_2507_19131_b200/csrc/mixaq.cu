@@ -46,10 +46,11 @@ void ctx_note(mixaq_ctx* ctx, const char* msg, int launches) {
 }  // namespace mixaq
 
 enum ProfCat { PC_ENERGY = 0, PC_SELECT, PC_LN1, PC_QKV, PC_ATTN, PC_PROJ, PC_LN2, PC_FC1, PC_FC2, PC_COPY,
-               PC_MERGE_GATHER, PC_MERGE_GEMM, PC_COUNT };
+               PC_MERGE_GATHER, PC_MERGE_GEMM, PC_STEM, PC_OUT_NORM, PC_COUNT };
 static const char* kProfNames[PC_COUNT] = {"energy", "select", "gather_ln1_quant", "gemm_qkv", "attention",
                                            "gemm_proj", "ln2_quant", "gemm_fc1_gelu", "gemm_fc2_scatter",
-                                           "copy_pruned", "merge_gather_ln_quant", "gemm_merge"};
+                                           "copy_pruned", "merge_gather_ln_quant", "gemm_merge", "patch_embed",
+                                           "stage_output_norm"};
 
 namespace {
 
@@ -280,7 +281,7 @@ mixaq_status mixaq_selftest_wait_timeout(mixaq_ctx* ctx, void* cuda_stream) {
 
 mixaq_status mixaq_measure_mma_peak(mixaq_ctx* ctx, int kind, int groups, void* scratch, size_t scratch_bytes,
                                     double* tera_ops_per_s, void* cuda_stream) {
-  if (!ctx || !scratch || !tera_ops_per_s || groups <= 0 || (kind != 0 && kind != 1)) return MIXAQ_INVALID_ARG;
+  if (!ctx || !scratch || !tera_ops_per_s || groups <= 0 || kind < 0 || kind > 2) return MIXAQ_INVALID_ARG;
   if (scratch_bytes < 1024 * sizeof(unsigned long long)) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "mma peak: scratch of 8 KiB needed");
   cudaStream_t st = (cudaStream_t)cuda_stream;
   unsigned long long* d_ns = (unsigned long long*)scratch;
@@ -291,8 +292,10 @@ mixaq_status mixaq_measure_mma_peak(mixaq_ctx* ctx, int kind, int groups, void* 
       cudaStreamSynchronize(st) != cudaSuccess) return check_cuda(ctx, "mma peak");
   unsigned long long worst = 1;
   for (auto v : ns) worst = v > worst ? v : worst;
-  // every SM issued groups x 4 MMAs of 128 x 256 x 32 multiply-accumulates; all SMs ran at once: the slowest one counts
-  const double ops = 2.0 * 128.0 * 256.0 * 32.0 * 4.0 * (double)groups * (double)sms;
+  // every SM issued groups x 4 MMAs of 128 x 256 x 32 (kind 2: x 64) multiply-accumulates; all SMs ran at once: the
+  // slowest one counts
+  const double k_per_mma = kind == 2 ? 64.0 : 32.0;
+  const double ops = 2.0 * 128.0 * 256.0 * k_per_mma * 4.0 * (double)groups * (double)sms;
   *tera_ops_per_s = ops / ((double)worst * 1e-9) / 1e12;
   return check_cuda(ctx, "mma peak");
 }
@@ -320,6 +323,25 @@ mixaq_status mixaq_profile_end(mixaq_ctx* ctx, void* cuda_stream, float* ms_per_
   }
   ctx->prof.clear();
   return check_cuda(ctx, "profile_end");
+}
+
+mixaq_status mixaq_profile_end_records(mixaq_ctx* ctx, void* cuda_stream, int* category, float* ms, int capacity, int* count) {
+  if (!ctx || !category || !ms || !count || capacity < 0) return MIXAQ_INVALID_ARG;
+  ctx->profiling = false;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return check_cuda(ctx, "profile_end_records");
+  int n = 0;
+  for (auto& r : ctx->prof) {
+    float t = 0.f;
+    if (n < capacity) {
+      if (cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess) { cudaGetLastError(); t = 0.f; }
+      category[n] = r.cat; ms[n] = t;
+    }
+    ++n;
+    ctx->pool.push_back(r.e0); ctx->pool.push_back(r.e1);
+  }
+  ctx->prof.clear();
+  *count = n;
+  return check_cuda(ctx, "profile_end_records");
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -416,6 +438,11 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     if (sel_out->cls)   cudaMemcpyAsync(sel_out->cls, sel.cls, n, cudaMemcpyDeviceToDevice, st);
     if (sel_out->order) cudaMemcpyAsync(sel_out->order, sel.order, n * 4, cudaMemcpyDeviceToDevice, st);
     if (sel_out->score) cudaMemcpyAsync(sel_out->score, sel.score, n * 8, cudaMemcpyDeviceToDevice, st);
+    if (sel_out->idx_hi || sel_out->idx_lo || sel_out->idx_pr) {
+      int32_t* const lists[3] = {sel_out->idx_hi, sel_out->idx_lo, sel_out->idx_pr};
+      const int cnt[3] = {g.n_hi, g.n_lo, g.n_pr};
+      launch_class_lists(sel.cls, B, g.nW, lists, cnt, st);
+    }
   }
 
   const mixaq_branch* brp[2] = {&p->hi, &p->lo};
@@ -563,11 +590,19 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
 
 // -------------------------------------------------------------------------------------------------
 namespace {
-struct BackboneWs { float* scratch; int32_t* energy; void* merge; void* block; char* sel; size_t merge_bytes, block_bytes, sel_bytes, bytes; };
-BackboneWs carve_backbone(const mixaq_backbone_params* p, int B, int H0, int W0, void* base) {
+struct BackboneWs {
+  float* scratch; int32_t* energy; void* merge; void* block; char* sel;
+  float* tokens;            // patch-embedding output (only with p->embed)
+  void* embed;              // patch-embedding workspace
+  float* raw[16];           // un-normalised stage maps (only with output norms)
+  size_t merge_bytes, block_bytes, sel_bytes, embed_bytes, bytes;
+};
+// H0, W0: size of the token map entering stage 1
+BackboneWs carve_backbone(const mixaq_backbone_params* p, int B, int H0, int W0, int Hi, int Wi, void* base) {
   BackboneWs w; Carver c(base);
   size_t max_map = 0, max_tok = 0, max_merge = 0, max_block = 0, max_sel = 0;
   int H = H0, W = W0, blk = 0;
+  const bool norms = p->out_norm_g && p->out_norm_b;
   for (int s = 0; s < p->num_stages; ++s) {
     if (s > 0) {
       max_merge = std::max(max_merge, mixaq_merge_workspace_bytes(&p->merges[s - 1], B, H, W));
@@ -579,21 +614,29 @@ BackboneWs carve_backbone(const mixaq_backbone_params* p, int B, int H0, int W0,
     for (int i = 0; i < p->depths[s]; ++i, ++blk)
       max_block = std::max(max_block, mixaq_block_workspace_bytes(&p->blocks[blk], B, H, W));
     max_sel = std::max(max_sel, (size_t)p->depths[s] * carve_sel(B, H, W, nullptr).bytes);   // one set per block of the stage
+    w.raw[s] = (norms && s < 16) ? c.take<float>((size_t)B * H * W * b0->dim) : nullptr;
   }
   w.scratch = c.take<float>(max_map);
   w.energy = c.take<int32_t>(max_tok);
   w.merge = c.take<uint8_t>(max_merge); w.merge_bytes = align_up(max_merge);
   w.block = c.take<uint8_t>(max_block); w.block_bytes = align_up(max_block);
   w.sel = (char*)c.take<uint8_t>(max_sel); w.sel_bytes = align_up(max_sel);
+  w.tokens = nullptr; w.embed = nullptr; w.embed_bytes = 0;
+  if (p->embed) {
+    w.tokens = c.take<float>((size_t)B * H0 * W0 * p->blocks[0].dim);
+    const size_t eb = mixaq_embed_workspace_bytes(p->embed, B, Hi, Wi);
+    w.embed = c.take<uint8_t>(eb); w.embed_bytes = align_up(eb);
+  }
   w.bytes = c.off;
   return w;
 }
 }  // namespace
 
 size_t mixaq_backbone_workspace_bytes(const mixaq_backbone_params* p, int B, int H0, int W0) {
-  if (!p || !p->depths || !p->blocks || p->num_stages <= 0 || B <= 0 || H0 <= 0 || W0 <= 0) return 0;
+  if (!p || !p->depths || !p->blocks || p->num_stages <= 0 || p->num_stages > 16 || B <= 0 || H0 <= 0 || W0 <= 0) return 0;
   if (p->num_stages > 1 && !p->merges) return 0;
-  return carve_backbone(p, B, H0, W0, nullptr).bytes;
+  const int Ht = p->embed ? (H0 + 3) / 4 : H0, Wt = p->embed ? (W0 + 3) / 4 : W0;
+  return carve_backbone(p, B, Ht, Wt, H0, W0, nullptr).bytes;
 }
 
 mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params* p, const float* x0,
@@ -605,6 +648,17 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     return fail(ctx, MIXAQ_INVALID_ARG, "backbone params incomplete");
   if (!x0 || !stage_out || !low_ratio_per_pair || !workspace || B <= 0 || H0 <= 0 || W0 <= 0)
     return fail(ctx, MIXAQ_INVALID_ARG, "backbone: bad argument");
+  if (p->num_stages > 16) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "at most 16 stages");
+  if ((p->out_norm_g != nullptr) != (p->out_norm_b != nullptr)) return fail(ctx, MIXAQ_INVALID_ARG, "output norms need gamma and beta");
+  const bool norms = p->out_norm_g && p->out_norm_b;
+  if (norms)
+    for (int s = 0; s < p->num_stages; ++s)
+      if (!p->out_norm_g[s] || !p->out_norm_b[s]) return fail(ctx, MIXAQ_INVALID_ARG, "output norm parameters of a stage are NULL");
+  if (p->embed && (!p->embed->prepared || p->embed->proj.out_features != p->blocks[0].dim))
+    return fail(ctx, MIXAQ_INVALID_ARG, "embed: not prepared, or its width differs from the first stage's");
+  // with a patch embedding in front, H0 x W0 is the image; the token map of stage 1 is a quarter of it
+  const int Hi = H0, Wi = W0;
+  if (p->embed) { H0 = (Hi + 3) / 4; W0 = (Wi + 3) / 4; }
   int nblk = 0;
   for (int s = 0; s < p->num_stages; ++s) {
     if (p->depths[s] <= 0 || (p->depths[s] != 1 && p->depths[s] % 2)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "depths must be even or 1");
@@ -617,7 +671,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     float r = low_ratio_per_pair[b / 2], q = prune_ratio_per_pair ? prune_ratio_per_pair[b / 2] : 0.f;
     if (!(r >= 0.f && r <= 1.f) || !(q >= 0.f && q <= 1.f)) return fail(ctx, MIXAQ_INVALID_ARG, "ratios must lie in [0, 1]");
   }
-  BackboneWs ws = carve_backbone(p, B, H0, W0, workspace);
+  BackboneWs ws = carve_backbone(p, B, H0, W0, Hi, Wi, workspace);
   if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "backbone workspace too small");
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
@@ -658,8 +712,16 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
       put(&q.ln_g, sizeof(q.ln_g)); put(&q.ln_b, sizeof(q.ln_b)); put_aq(q.in); put_lin(q.reduction);
       put(&q.prepared, sizeof(q.prepared));
     }
+    const char has_embed = p->embed ? 1 : 0, has_norms = norms ? 1 : 0;
+    put(&has_embed, 1); put(&has_norms, 1);
+    if (p->embed) {
+      const mixaq_embed_params& q = *p->embed;
+      put(&q.ln_g, sizeof(q.ln_g)); put(&q.ln_b, sizeof(q.ln_b)); put(&q.bias, sizeof(q.bias)); put_aq(q.in); put_lin(q.proj);
+      put(&q.prepared, sizeof(q.prepared));
+    }
+    if (norms) { put(p->out_norm_g, sizeof(float*) * p->num_stages); put(p->out_norm_b, sizeof(float*) * p->num_stages); }
     put(&x0, sizeof(x0)); put(stage_out, sizeof(float*) * p->num_stages);
-    const int dims[3] = {B, H0, W0}; put(dims, sizeof(dims));
+    const int dims[5] = {B, H0, W0, Hi, Wi}; put(dims, sizeof(dims));
     put(low_ratio_per_pair, sizeof(float) * npairs);
     const char has_prune = prune_ratio_per_pair ? 1 : 0; put(&has_prune, 1);
     if (prune_ratio_per_pair) put(prune_ratio_per_pair, sizeof(float) * npairs);
@@ -677,9 +739,17 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   mixaq_status result = MIXAQ_OK;
   int total = 0, H = H0, W = W0, blk = 0;
   const float* cur = x0;
+  if (p->embed) {
+    // image -> token map of stage 1 (patch embedding), inside the same captured graph
+    result = mixaq_embed_forward(ctx, p->embed, x0, ws.tokens, B, Hi, Wi, ws.embed, ws.embed_bytes, st);
+    total += ctx->launches;
+    cur = ws.tokens;
+  }
   for (int s = 0; s < p->num_stages && result == MIXAQ_OK; ++s) {
     const int d = p->depths[s];
-    float* out_s = stage_out[s];
+    // with output norms the un-normalised map stays in the workspace (the next stage reads it) and the caller's
+    // buffer receives its LayerNorm
+    float* out_s = norms ? ws.raw[s] : stage_out[s];
     if (s > 0) {
       // the merge writes where the first block of the stage does NOT write
       float* mdst = (d % 2 == 0) ? out_s : ws.scratch;
@@ -723,6 +793,13 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
       if (result != MIXAQ_OK) break;
       total += ctx->launches;
       cur = dst;
+    }
+    if (result == MIXAQ_OK && norms) {
+      PROF(PC_OUT_NORM);
+      g_launches = 0;
+      if (!launch_bias_ln(out_s, nullptr, p->out_norm_g[s], p->out_norm_b[s], stage_out[s], (long)B * H * W, b0->dim, st))
+        result = fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "output norm: unsupported width");
+      total += g_launches;
     }
   }
   if (use_graph) {
@@ -802,6 +879,7 @@ mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, co
   EmbedPrepared pr = carve_embed(p, p->prepared);
   g_launches = 0;
   PatchGatherArgs pg; pg.img = image; pg.out = codes; pg.q = to_aq(p->in); pg.B = B; pg.Hi = Hi; pg.Wi = Wi;
+  PROF(PC_STEM);
   launch_patch_gather(pg, st);
   GemmArgs ga;
   ga.status = ctx->d_status;

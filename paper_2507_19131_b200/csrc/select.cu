@@ -102,6 +102,33 @@ __global__ void __launch_bounds__(RANK_WARPS * 32) k_rank_emit(const __grid_cons
   for (int t = lane; t < WT; t += 32) dst[slot * WT + t] = window_src(b, a.H, a.W, Hp, Wp, a.shift, a.nwx, w, t);
 }
 
+// One warp per (image, class): walks the windows in ascending index, 32 at a time, and appends the members of its class
+// (order-preserving compaction by ballot).
+struct ClassListArgs { const uint8_t* cls; int32_t* out[3]; int count[3]; int B, nW; };
+__global__ void __launch_bounds__(96) k_class_lists(ClassListArgs a) {
+  const int b = blockIdx.x, c = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int32_t* out = a.out[c];
+  if (!out) return;
+  out += (long)b * a.count[c];
+  const uint8_t* cls = a.cls + (long)b * a.nW;
+  int base = 0;
+  for (int w0 = 0; w0 < a.nW; w0 += 32) {
+    const int w = w0 + lane;
+    const bool mine = w < a.nW && cls[w] == c;
+    const unsigned m = __ballot_sync(0xffffffffu, mine);
+    if (mine) out[base + __popc(m & ((1u << lane) - 1u))] = w;
+    base += __popc(m);
+  }
+}
+
+void launch_class_lists(const uint8_t* cls, int B, int nW, int32_t* const out[3], const int count[3], cudaStream_t st) {
+  ClassListArgs a;
+  a.cls = cls; a.B = B; a.nW = nW;
+  for (int c = 0; c < 3; ++c) { a.out[c] = out[c]; a.count[c] = count[c]; }
+  k_class_lists<<<B, 96, 0, st>>>(a);
+  ++g_launches;
+}
+
 void launch_energy(const float* x, int32_t* energy, long ntok, int C, float inv_scale, cudaStream_t st) {
   k_energy<<<(unsigned)((ntok * 8 + 255) / 256), 256, 0, st>>>(x, energy, ntok, C, inv_scale);
   ++g_launches;

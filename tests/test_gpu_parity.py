@@ -73,6 +73,11 @@ def run_block_case(orc, mq, ctx, blk, x, low, prune=0.0, reverse=False, stage_en
     assert np.array_equal(got.scores.cpu().numpy(), ref.scores)
     assert np.array_equal(got.order.cpu().numpy(), ref.order)
     assert np.array_equal(got.cls.cpu().numpy(), ref.cls)
+    # per-class window lists in ascending window index: what is unique given the classes
+    for c, lst in enumerate((got.idx_hi, got.idx_lo, got.idx_pr)):
+        lst = lst.cpu().numpy()
+        for b in range(x.shape[0]):
+            assert np.array_equal(lst[b], np.flatnonzero(ref.cls[b] == c)), f"class {c} list of image {b}"
     if taps:
         check_taps(orc, blk, ref, got, ref.counts)
     y = got.y.cpu().numpy()
@@ -334,6 +339,31 @@ def test_image_to_normed_stage_maps_end_to_end(orc, mq, ctx):
         assert np.array_equal(gg, ww)
 
 
+def test_image_to_normed_stage_maps_in_one_backbone_call(orc, mq, ctx):
+    """The same chain through ONE mixaq_backbone_forward call (stem and output norms given in the backbone parameters),
+    on a capturable stream: first call captures the graph, second replays it."""
+    wl = synth.tiny_backbone(ratio=0.4, prune=0.2)
+    rng = np.random.default_rng(13)
+    e = synth.make_embed(rng, wl.backbone.dims[0])
+    Hi, Wi = 4 * wl.H - 1, 4 * wl.W - 2
+    img = synth.input_image(14, wl.B, Hi, Wi)
+    norms = [((1.0 + 0.05 * rng.standard_normal(c)).astype(F32), (0.05 * rng.standard_normal(c)).astype(F32)) for c in wl.backbone.dims]
+    x0_ref = orc.patch_embed(e, img)
+    want = [orc.layernorm(o, g, b) for o, (g, b) in zip(orc.backbone_forward(wl.backbone, x0_ref, wl.low_ratios, wl.prune_ratios), norms)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, Hi, Wi, embed=e, norms=norms)
+        imd = dev(img)
+        for call in range(2):
+            got = mq.backbone_forward(ctx, dbb, imd, wl.low_ratios, wl.prune_ratios)
+            side.synchronize()
+            for st, (g, w) in enumerate(zip(got, want)):
+                assert np.array_equal(g.cpu().numpy(), w), f"stage {st}, call {call}"
+    torch.cuda.current_stream().wait_stream(side)
+    assert ctx.device_status() == 0
+
+
 def test_bounded_wait_runs_out_and_the_context_stays_usable(orc, mq):
     """Failure path without a fault: a barrier that nothing signals makes the kernels' bounded wait run out; the status
     word reports it, can be cleared, and the next forward on the same context is correct."""
@@ -371,13 +401,16 @@ def test_calibration_on_the_gpu_feeds_the_quantized_forward(orc, mq, ctx):
 
 
 def test_mma_issue_rate_microbenchmark(mq, ctx):
-    """The library's own tensor-core loop: kind::i8 reaches petaops, and kind::f8f6f4 (the path of the 4/6-bit operand
-    formats) is not faster, which is why the low branch keeps using kind::i8."""
+    """The library's own tensor-core loop: kind::i8 reaches petaops; kind::f8f6f4 (the path of the 4/6-bit operand
+    formats in 8-bit containers) is not faster; kind::mxf4 (block-scaled E2M1, the one narrower path with a higher
+    nominal rate) is measured next to them.  The numbers behind the choice of kind::i8 for the low-bit branch."""
     i8 = ctx.measure_mma_peak(0, 2000)
     f8 = ctx.measure_mma_peak(1, 2000)
+    mx = ctx.measure_mma_peak(2, 2000)
     assert ctx.device_status() == 0
-    assert 1500.0 < i8 < 6000.0 and 1500.0 < f8 < 6000.0
+    assert 1500.0 < i8 < 6000.0 and 1500.0 < f8 < 6000.0 and 1500.0 < mx < 12000.0
     assert f8 < 1.1 * i8
+    print(f"mma issue rate TOP/s: i8 {i8:.0f}  f8f6f4 {f8:.0f}  mxf4 {mx:.0f}")
 
 
 def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
