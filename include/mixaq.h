@@ -206,6 +206,29 @@ mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, co
 mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float* beta, const float* x, float* y,
                                 long rows, int C, void* cuda_stream);
 
+/* ---- calibration of the activation quantizers (Section 4.3, post-training flow): one calibration sample, and the
+ *      FULL feature map (every window, whatever branch it will later run in) sets the ranges of BOTH branches, which
+ *      then differ only in bit width.  mixaq_calibrate_block runs the floating-point block (all quantizers off,
+ *      weights = code x step size) with every window through the LayerNorm parameters and biases of one branch
+ *      (branch 0: high, 1: low), writes its output map to y and the minimum / maximum each quantizer site saw to
+ *      `ranges` (a HOST struct).  The quantizer fields of `p` are not read and `p->prepared` is not needed.
+ *      mixaq_calibrate_merge does the same for a patch merging (one site: the LayerNorm output).
+ *      Both synchronise the stream.  mixaq_aq_from_range is the one definition of the quantizer that covers a range:
+ *      scale = (hi - lo) / (2^bits - 1), inv_scale = 1 / scale, zero_point = clamp(rne(-lo / scale), 0, 2^bits - 1). ---- */
+typedef struct { float lo, hi; } mixaq_range;
+typedef struct { mixaq_range qkv_in, q, k, v, proj_in, fc1_in, fc2_in;
+                 mixaq_range x_in;   /* the block's input map itself (its largest magnitude sets the score-code step) */
+               } mixaq_block_ranges;
+size_t       mixaq_calibrate_block_workspace_bytes(const mixaq_block_params* p, int B, int H, int W);
+mixaq_status mixaq_calibrate_block(mixaq_ctx* ctx, const mixaq_block_params* p, int branch, const float* x, float* y,
+                                   int B, int H, int W, mixaq_block_ranges* ranges,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t       mixaq_calibrate_merge_workspace_bytes(const mixaq_merge_params* p, int B, int H, int W);
+mixaq_status mixaq_calibrate_merge(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
+                                   int B, int H, int W, mixaq_range* range,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+mixaq_status mixaq_aq_from_range(float lo, float hi, int bits, mixaq_aq* out);
+
 /* ---- the backbone: for every stage [merge] -> stage energy -> blocks; one ratio per pair of consecutive
  *      blocks (Section 3.3), optional prune ratio per pair (Section 3.4).  x0 is the [B][H0][W0][C0] map after the
  *      patch-embedding stem (or, when p->embed is set, the [B][H0][W0][3] image itself); stage_out is a HOST array of

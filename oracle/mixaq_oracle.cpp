@@ -285,15 +285,26 @@ void fp_linear(const float* a, int M, int K, const orc_linear& L, const float* b
     }
 }
 
+// ranges (optional): 7 x {min, max} of what the quantizers of the sites QKV input, q, k, v, proj input, fc1 input,
+// fc2 input would see, over every row of the window (pad rows included: they pass through the layers like any row)
+struct SiteRanges { float lo[7], hi[7]; };
+inline void observe(SiteRanges* r, int site, const float* v, long n) {
+  if (!r) return;
+  for (long i = 0; i < n; ++i) { r->lo[site] = std::fmin(r->lo[site], v[i]); r->hi[site] = std::fmax(r->hi[site], v[i]); }
+}
+
 void window_forward_fp(const orc_block& P, const orc_branch& br, const float* relb, const float* mask,
-                       const float* xin, const uint8_t* real, float* yout) {
+                       const float* xin, const uint8_t* real, float* yout, SiteRanges* rng = nullptr) {
   const int C = P.dim, T = P.window * P.window, nh = P.heads, d = C / nh, Hd = P.hidden;
   std::vector<float> ln((long)T * C), qkv((long)T * 3 * C), o((long)T * C), po((long)T * C), x1((long)T * C);
   for (int t = 0; t < T; ++t) {
     if (real[t]) layernorm_row(xin + (long)t * C, C, br.ln1_g, br.ln1_b, &ln[(long)t * C]);
     else std::fill(&ln[(long)t * C], &ln[(long)(t + 1) * C], 0.0f);
   }
+  observe(rng, 0, ln.data(), (long)T * C);
   fp_linear(ln.data(), T, C, P.qkv, br.b_qkv, qkv.data());
+  for (int t = 0; t < T; ++t)
+    for (int sec = 0; sec < 3; ++sec) observe(rng, 1 + sec, &qkv[(long)t * 3 * C + sec * C], C);
   std::vector<float> logits(T), prob(T);
   const double rs = 1.0 / std::sqrt((double)d);
   for (int h = 0; h < nh; ++h)
@@ -310,19 +321,22 @@ void window_forward_fp(const orc_block& P, const orc_branch& br, const float* re
         o[(long)i * C + h * d + e] = (float)s;
       }
     }
+  observe(rng, 4, o.data(), (long)T * C);
   fp_linear(o.data(), T, C, P.proj, br.b_proj, po.data());
   for (long e = 0; e < (long)T * C; ++e) x1[e] = xin[e] + po[e];
   for (int t = 0; t < T; ++t) layernorm_row(&x1[(long)t * C], C, br.ln2_g, br.ln2_b, &ln[(long)t * C]);
+  observe(rng, 5, ln.data(), (long)T * C);
   std::vector<float> h1((long)T * Hd), h2((long)T * C);
   fp_linear(ln.data(), T, C, P.fc1, br.b_fc1, h1.data());
   for (auto& v : h1) v = gelu1(v);
+  observe(rng, 6, h1.data(), (long)T * Hd);
   fp_linear(h1.data(), T, Hd, P.fc2, br.b_fc2, h2.data());
   for (long e = 0; e < (long)T * C; ++e) yout[e] = x1[e] + h2[e];
 }
 
 // gather one window's tokens (pad -> zeros), run it, scatter the real tokens back
 void run_window(const orc_block& P, const orc_branch& br, const float* relb, const float* x, float* y,
-                int img, int H, int W, int w, const WinTaps* wt) {
+                int img, int H, int W, int w, const WinTaps* wt, SiteRanges* rng = nullptr) {
   const int C = P.dim, ws = P.window, T = ws * ws;
   std::vector<float> xin((long)T * C, 0.0f), yout((long)T * C);
   std::vector<uint8_t> real(T);
@@ -336,7 +350,7 @@ void run_window(const orc_block& P, const orc_branch& br, const float* relb, con
   if (P.shift > 0) { mask.resize((long)T * T); shift_mask(H, W, ws, P.shift, w, mask.data()); }
   const float* mk = P.shift > 0 ? mask.data() : nullptr;
   if (P.quant) window_forward_quant(P, br, relb, mk, xin.data(), real.data(), yout.data(), wt);
-  else         window_forward_fp(P, br, relb, mk, xin.data(), real.data(), yout.data());
+  else         window_forward_fp(P, br, relb, mk, xin.data(), real.data(), yout.data(), rng);
   for (int t = 0; t < T; ++t)
     if (real[t]) std::memcpy(y + ((long)img * H * W + src[t]) * C, &yout[(long)t * C], C * sizeof(float));
 }
@@ -599,6 +613,52 @@ void orc_uniform_block_forward(const orc_block* p, const orc_branch* br, const f
 #pragma omp parallel for schedule(dynamic, 4)
   for (long job = 0; job < (long)B * nW; ++job)
     run_window(P, *br, relb.data(), x, y, (int)(job / nW), H, W, (int)(job % nW), nullptr);
+}
+
+// Calibration observer (Section 4.3: the full feature map calibrates both branches): the floating-point block
+// (quantizers off, whatever P.quant says) with every window through the LayerNorm parameters and biases of `br`;
+// y = its output, ranges[2*site], ranges[2*site+1] = min, max seen at the seven quantizer sites (order: QKV input, q,
+// k, v, proj input, fc1 input, fc2 input) over all rows of all windows.
+void orc_block_observe_fp(const orc_block* p, const orc_branch* br, const float* x, float* y, int B, int H, int W,
+                          float* ranges /* [14] */) {
+  orc_block P = *p;
+  P.quant = 0;
+  const int ws = P.window, T = ws * ws;
+  const int Hp = round_up(H, ws), Wp = round_up(W, ws), nW = (Hp / ws) * (Wp / ws);
+  std::vector<float> relb((long)P.heads * T * T);
+  relpos_bias(P.relpos, ws, P.heads, relb.data());
+  SiteRanges all;
+  for (int i = 0; i < 7; ++i) { all.lo[i] = INFINITY; all.hi[i] = -INFINITY; }
+#pragma omp parallel
+  {
+    SiteRanges mine = all;
+#pragma omp for schedule(dynamic, 4)
+    for (long job = 0; job < (long)B * nW; ++job)
+      run_window(P, *br, relb.data(), x, y, (int)(job / nW), H, W, (int)(job % nW), nullptr, &mine);
+#pragma omp critical
+    for (int i = 0; i < 7; ++i) { all.lo[i] = std::fmin(all.lo[i], mine.lo[i]); all.hi[i] = std::fmax(all.hi[i], mine.hi[i]); }
+  }
+  for (int i = 0; i < 7; ++i) { ranges[2 * i] = all.lo[i]; ranges[2 * i + 1] = all.hi[i]; }
+}
+
+// the same for patch merging: min, max of the LayerNorm output that the merge's input quantizer would see
+void orc_merge_observe_fp(const orc_merge* m, const float* x, int B, int H, int W, int C, float* y, float* range /* [2] */) {
+  const int H2 = (H + 1) / 2, W2 = (W + 1) / 2, K = 4 * C, N = m->red.out_f;
+  float lo = INFINITY, hi = -INFINITY;
+  for (long tok = 0; tok < (long)B * H2 * W2; ++tok) {
+    int b = (int)(tok / ((long)H2 * W2)), r = (int)(tok % ((long)H2 * W2));
+    int y2 = r / W2, x2 = r % W2;
+    std::vector<float> cat(K, 0.0f), ln(K);
+    const int dy[4] = {0, 1, 0, 1}, dx[4] = {0, 0, 1, 1};
+    for (int g = 0; g < 4; ++g) {
+      int yy = 2 * y2 + dy[g], xx = 2 * x2 + dx[g];
+      if (yy < H && xx < W) std::memcpy(&cat[(long)g * C], x + (((long)b * H + yy) * W + xx) * C, C * sizeof(float));
+    }
+    layernorm_row(cat.data(), K, m->ln_g, m->ln_b, ln.data());
+    for (int k = 0; k < K; ++k) { lo = std::fmin(lo, ln[k]); hi = std::fmax(hi, ln[k]); }
+    fp_linear(ln.data(), 1, K, m->red, nullptr, y + tok * N);
+  }
+  range[0] = lo; range[1] = hi;
 }
 
 // patch merging: 2x2 neighbours concatenated (zero-padded when H or W is odd) -> LN(4C) -> quantize ->

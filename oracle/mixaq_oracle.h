@@ -111,6 +111,13 @@ void  orc_block_forward(const orc_block* p, const float* x, float* y, int B, int
 void  orc_uniform_block_forward(const orc_block* p, const orc_branch* br, const float* x, float* y,
                                 int B, int H, int W);
 void  orc_merge_forward(const orc_merge* m, const float* x, int B, int H, int W, int C, float* y);
+/* Calibration observers (Section 4.3: one sample, the FULL feature map calibrates both branches): the floating-point
+ * block / merge (quantizers off) and the min, max each quantizer site would see.  ranges = 7 x {min, max} in the order
+ * QKV input, q, k, v, proj input, fc1 input, fc2 input, over all rows of all windows (pad rows included).  Pinned in
+ * the tests to a textbook block written on the un-windowed map in binary64. */
+void  orc_block_observe_fp(const orc_block* p, const orc_branch* br, const float* x, float* y, int B, int H, int W,
+                           float* ranges /* [14] */);
+void  orc_merge_observe_fp(const orc_merge* m, const float* x, int B, int H, int W, int C, float* y, float* range /* [2] */);
 /* blocks: sum(depths) entries; merges: num_stages-1; stage_out: num_stages buffers [B][Hs][Ws][Cs] */
 void  orc_backbone_forward(int num_stages, const int* depths, const orc_block* blocks, const orc_merge* merges,
                            const float* x0, float* const* stage_out, int B, int H0, int W0,

@@ -308,6 +308,33 @@ def uniform_block_forward(blk, branch_name, x, quant=True):
     return y
 
 
+SITES = ("qkv_in", "q", "k", "v", "proj_in", "fc1_in", "fc2_in")
+
+
+def block_observe_fp(blk, branch_name, x):
+    """Floating-point block through one branch's LayerNorm parameters and biases; returns (y, {site: (min, max)})."""
+    x = np.ascontiguousarray(x, np.float32)
+    B, H, W, _ = x.shape
+    keep = _Keep()
+    bs = block_struct(keep, blk, quant=False)
+    br = bs.hi if branch_name == "hi" else bs.lo
+    y = np.empty_like(x)
+    r = np.empty(14, np.float32)
+    lib().orc_block_observe_fp(C.byref(bs), C.byref(br), _p(x), _p(y), B, H, W, _p(r))
+    return y, {s: (float(r[2 * i]), float(r[2 * i + 1])) for i, s in enumerate(SITES)}
+
+
+def merge_observe_fp(m, x):
+    x = np.ascontiguousarray(x, np.float32)
+    B, H, W, Cc = x.shape
+    keep = _Keep()
+    ms = merge_struct(keep, m, quant=False)
+    y = np.empty((B, (H + 1) // 2, (W + 1) // 2, m.red.codes.shape[0]), np.float32)
+    r = np.empty(2, np.float32)
+    lib().orc_merge_observe_fp(C.byref(ms), _p(x), B, H, W, Cc, _p(y), _p(r))
+    return y, (float(r[0]), float(r[1]))
+
+
 def merge_forward(m, x, quant=True):
     x = np.ascontiguousarray(x, np.float32)
     B, H, W, Cc = x.shape

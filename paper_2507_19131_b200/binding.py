@@ -23,7 +23,8 @@ EXPORTS = [
     "mixaq_backbone_forward", "mixaq_last_launch_count", "mixaq_profile_categories", "mixaq_profile_category_name",
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
-    "mixaq_norm_forward", "mixaq_profile_end_records", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
+    "mixaq_norm_forward", "mixaq_profile_end_records", "mixaq_calibrate_block_workspace_bytes", "mixaq_calibrate_block",
+    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -113,7 +114,8 @@ def lib():
         L.mixaq_profile_category_name.restype = C.c_char_p
         for n in ("mixaq_embed_prepared_bytes", "mixaq_embed_workspace_bytes",
                   "mixaq_block_prepared_bytes", "mixaq_merge_prepared_bytes", "mixaq_block_workspace_bytes",
-                  "mixaq_merge_workspace_bytes", "mixaq_backbone_workspace_bytes"):
+                  "mixaq_merge_workspace_bytes", "mixaq_backbone_workspace_bytes",
+                  "mixaq_calibrate_block_workspace_bytes", "mixaq_calibrate_merge_workspace_bytes"):
             getattr(L, n).restype = C.c_size_t
         L.mixaq_low_count.argtypes = [C.c_float, C.c_int]
         _lib = L
@@ -402,6 +404,53 @@ def norm_forward(ctx: Context, gamma: torch.Tensor, beta: torch.Tensor, x: torch
     ctx.check(lib().mixaq_norm_forward(ctx.h, _ptr(gamma), _ptr(beta), _ptr(x), _ptr(y), C.c_long(x.numel() // Cc), Cc,
                                        _stream_ptr()), "norm_forward")
     return y
+
+
+class RangeS(C.Structure):
+    _fields_ = [("lo", C.c_float), ("hi", C.c_float)]
+
+
+CAL_SITES = ("qkv_in", "q", "k", "v", "proj_in", "fc1_in", "fc2_in", "x_in")
+
+
+class BlockRangesS(C.Structure):
+    _fields_ = [(n, RangeS) for n in CAL_SITES]
+
+
+def aq_from_range(lo: float, hi: float, bits: int):
+    """mixaq_aq_from_range: the quantizer of `bits` bits that covers [lo, hi]; returns (scale, inv_scale, zero_point)."""
+    q = AQ()
+    st = lib().mixaq_aq_from_range(C.c_float(lo), C.c_float(hi), bits, C.byref(q))
+    if st != 0:
+        raise MixaqError(st, "aq_from_range")
+    return float(q.scale), float(q.inv_scale), int(q.zero_point)
+
+
+def calibrate_block(ctx: Context, block_struct: BlockS, branch: int, x: torch.Tensor, y: torch.Tensor = None):
+    """mixaq_calibrate_block: floating-point block through one branch (0 high, 1 low) with the min/max observers.
+    Returns (y, {site: (lo, hi)})."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    B, H, W, _ = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    need = lib().mixaq_calibrate_block_workspace_bytes(C.byref(block_struct), B, H, W)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    r = BlockRangesS()
+    ctx.check(lib().mixaq_calibrate_block(ctx.h, C.byref(block_struct), branch, _ptr(x), _ptr(y), B, H, W, C.byref(r),
+                                          _ptr(ws), C.c_size_t(ws.numel()), _stream_ptr()), "calibrate_block")
+    return y, {n: (float(getattr(r, n).lo), float(getattr(r, n).hi)) for n in CAL_SITES}
+
+
+def calibrate_merge(ctx: Context, merge_struct: MergeS, x: torch.Tensor):
+    """mixaq_calibrate_merge: floating-point patch merging; returns (y, (lo, hi)) of its LayerNorm output."""
+    B, H, W, Cc = x.shape
+    y = torch.empty((B, (H + 1) // 2, (W + 1) // 2, 2 * Cc), dtype=torch.float32, device=x.device)
+    need = lib().mixaq_calibrate_merge_workspace_bytes(C.byref(merge_struct), B, H, W)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    r = RangeS()
+    ctx.check(lib().mixaq_calibrate_merge(ctx.h, C.byref(merge_struct), _ptr(x), _ptr(y), B, H, W, C.byref(r), _ptr(ws),
+                                          C.c_size_t(ws.numel()), _stream_ptr()), "calibrate_merge")
+    return y, (float(r.lo), float(r.hi))
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -105,6 +105,26 @@ struct AttnArgs {
 };
 void launch_attention(const AttnArgs& a, cudaStream_t st);
 
+// ---- calibration: floating-point block / merge with min-max observers at the quantizer sites -----------------------
+struct CalBlockArgs {
+  const float* x; float* y;                       // feature maps [B][H][W][C]
+  int B, H, W, C, heads, hidden, shift;
+  const float *ln1_g, *ln1_b, *ln2_g, *ln2_b, *b_qkv, *b_proj, *b_fc1, *b_fc2;   // of the branch being calibrated
+  const int8_t *w_qkv, *w_proj, *w_fc1, *w_fc2;
+  const float *s_qkv, *s_proj, *s_fc1, *s_fc2, *relpos;
+  int32_t* rowsrc; float *ln, *qkv, *o, *x1, *h;  // workspace: [M], [M][C], [M][3C], [M][C], [M][C], [M][hidden]
+  uint32_t* obs;                                  // 16 order-preserving keys: min, max of the seven sites and of x
+};
+bool launch_calibrate_block(const CalBlockArgs& c, cudaStream_t st);
+struct CalMergeArgs {
+  const float* x; float* y; int B, H, W, C, N;
+  const float *ln_g, *ln_b; const int8_t* w; const float* sw;
+  float* ln;                                      // workspace [M][4C]
+  uint32_t* obs;                                  // 2 keys
+};
+bool launch_calibrate_merge(const CalMergeArgs& c, cudaStream_t st);
+float cal_key_to_float(uint32_t key);
+
 // ---- preparation -----------------------------------------------------------------------------------
 void launch_prepare_linear(const int8_t* w, const float* sw, int N, int K, float sa, int za, float* mult,
                            int32_t* zc, cudaStream_t st);

@@ -112,7 +112,12 @@ bool branch_ok(const mixaq_branch& b) {
          aq_ok(b.proj_in, b.bits) && aq_ok(b.fc1_in, b.bits) && aq_ok(b.fc2_in, b.bits);
 }
 
-mixaq_status validate_block(mixaq_ctx* ctx, const mixaq_block_params* p) {
+bool branch_ptrs_ok(const mixaq_branch& b) {
+  return b.ln1_g && b.ln1_b && b.ln2_g && b.ln2_b && b.b_qkv && b.b_proj && b.b_fc1 && b.b_fc2;
+}
+
+// need_quantizers = false: the calibration pass, which runs before any quantizer exists
+mixaq_status validate_block(mixaq_ctx* ctx, const mixaq_block_params* p, bool need_quantizers = true) {
   if (!p) return fail(ctx, MIXAQ_INVALID_ARG, "block params are NULL");
   if (p->window != WS) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "window must be 7");
   if (p->dim <= 0 || p->dim % 32 || !ln_dim_supported(p->dim)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "unsupported dim");
@@ -123,6 +128,10 @@ mixaq_status validate_block(mixaq_ctx* ctx, const mixaq_block_params* p) {
       !linear_ok(p->fc1, p->hidden, p->dim) || !linear_ok(p->fc2, p->dim, p->hidden))
     return fail(ctx, MIXAQ_INVALID_ARG, "weight matrix missing or of the wrong shape");
   if (!p->relpos_table) return fail(ctx, MIXAQ_INVALID_ARG, "relpos_table is NULL");
+  if (!need_quantizers) {
+    if (!branch_ptrs_ok(p->hi) || !branch_ptrs_ok(p->lo)) return fail(ctx, MIXAQ_INVALID_ARG, "branch parameters invalid");
+    return MIXAQ_OK;
+  }
   if (!branch_ok(p->hi) || !branch_ok(p->lo)) return fail(ctx, MIXAQ_INVALID_ARG, "branch parameters invalid");
   if (!(p->score_inv_scale > 0.f)) return fail(ctx, MIXAQ_INVALID_ARG, "score_inv_scale must be positive");
   return MIXAQ_OK;
@@ -923,6 +932,105 @@ mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled) {
     for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
     ctx->graphs.clear();
   }
+  return MIXAQ_OK;
+}
+
+// -------------------------------------------------------------------------------------------------
+// calibration (Section 4.3)
+namespace {
+struct CalWs { int32_t* rowsrc; float *ln, *qkv, *o, *x1, *h; uint32_t* obs; size_t bytes; };
+CalWs carve_cal(const mixaq_block_params* p, int B, int H, int W, void* base) {
+  CalWs w; Carver c(base);
+  Geometry g = geometry(H, W, 0.f, 0.f);
+  const size_t M = (size_t)B * g.nW * WT;
+  w.obs = c.take<uint32_t>(16);
+  w.rowsrc = c.take<int32_t>(M);
+  w.ln = c.take<float>(M * p->dim); w.qkv = c.take<float>(M * 3 * p->dim); w.o = c.take<float>(M * p->dim);
+  w.x1 = c.take<float>(M * p->dim); w.h = c.take<float>(M * p->hidden);
+  w.bytes = c.off;
+  return w;
+}
+// reads the observers' keys back (synchronises) and decodes them
+mixaq_status read_ranges(mixaq_ctx* ctx, const uint32_t* d_obs, int sites, mixaq_range* out, cudaStream_t st) {
+  uint32_t keys[16];
+  if (cudaMemcpyAsync(keys, d_obs, sizeof(uint32_t) * 2 * sites, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) return check_cuda(ctx, "calibrate (read ranges)") == MIXAQ_OK ? MIXAQ_CUDA_ERROR : MIXAQ_CUDA_ERROR;
+  for (int i = 0; i < sites; ++i) { out[i].lo = cal_key_to_float(keys[2 * i]); out[i].hi = cal_key_to_float(keys[2 * i + 1]); }
+  return MIXAQ_OK;
+}
+}  // namespace
+
+size_t mixaq_calibrate_block_workspace_bytes(const mixaq_block_params* p, int B, int H, int W) {
+  if (!p || B <= 0 || H <= 0 || W <= 0 || p->dim <= 0 || p->hidden <= 0) return 0;
+  return carve_cal(p, B, H, W, nullptr).bytes;
+}
+
+mixaq_status mixaq_calibrate_block(mixaq_ctx* ctx, const mixaq_block_params* p, int branch, const float* x, float* y,
+                                   int B, int H, int W, mixaq_block_ranges* ranges,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  mixaq_status s = validate_block(ctx, p, false);
+  if (s != MIXAQ_OK) return s;
+  if (!x || !y || x == y || !ranges || !workspace || B <= 0 || H <= 0 || W <= 0 || (branch != 0 && branch != 1))
+    return fail(ctx, MIXAQ_INVALID_ARG, "calibrate_block: bad argument");
+  if ((long)B * H * W >= (1L << 31) / WT) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many tokens");
+  CalWs ws = carve_cal(p, B, H, W, workspace);
+  if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "calibrate_block workspace too small");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const mixaq_branch& br = branch == 0 ? p->hi : p->lo;
+  CalBlockArgs c;
+  c.x = x; c.y = y; c.B = B; c.H = H; c.W = W; c.C = p->dim; c.heads = p->heads; c.hidden = p->hidden; c.shift = p->shift;
+  c.ln1_g = br.ln1_g; c.ln1_b = br.ln1_b; c.ln2_g = br.ln2_g; c.ln2_b = br.ln2_b;
+  c.b_qkv = br.b_qkv; c.b_proj = br.b_proj; c.b_fc1 = br.b_fc1; c.b_fc2 = br.b_fc2;
+  c.w_qkv = p->qkv.codes; c.w_proj = p->proj.codes; c.w_fc1 = p->fc1.codes; c.w_fc2 = p->fc2.codes;
+  c.s_qkv = p->qkv.scale; c.s_proj = p->proj.scale; c.s_fc1 = p->fc1.scale; c.s_fc2 = p->fc2.scale; c.relpos = p->relpos_table;
+  c.rowsrc = ws.rowsrc; c.ln = ws.ln; c.qkv = ws.qkv; c.o = ws.o; c.x1 = ws.x1; c.h = ws.h; c.obs = ws.obs;
+  g_launches = 0;
+  if (!launch_calibrate_block(c, st)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "calibrate_block: unsupported dim");
+  ctx->launches = g_launches;
+  s = check_cuda(ctx, "calibrate_block");
+  if (s != MIXAQ_OK) return s;
+  return read_ranges(ctx, ws.obs, 8, &ranges->qkv_in, st);
+}
+
+size_t mixaq_calibrate_merge_workspace_bytes(const mixaq_merge_params* p, int B, int H, int W) {
+  if (!p || B <= 0 || H <= 0 || W <= 0 || p->reduction.in_features <= 0) return 0;
+  const size_t toks = (size_t)B * ((H + 1) / 2) * ((W + 1) / 2);
+  return align_up(16 * sizeof(uint32_t)) + align_up(toks * p->reduction.in_features * sizeof(float));
+}
+
+mixaq_status mixaq_calibrate_merge(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,
+                                   int B, int H, int W, mixaq_range* range,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !p) return MIXAQ_INVALID_ARG;
+  if (!x || !y || !range || !workspace || B <= 0 || H <= 0 || W <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "calibrate_merge: bad argument");
+  const int K = p->reduction.in_features, N = p->reduction.out_features, C = K / 4;
+  if (K % 4 || N <= 0 || !merge_dim_supported(C)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "calibrate_merge: unsupported dims");
+  if (!p->ln_g || !p->ln_b || !p->reduction.codes || !p->reduction.scale) return fail(ctx, MIXAQ_INVALID_ARG, "merge params incomplete");
+  if (mixaq_calibrate_merge_workspace_bytes(p, B, H, W) > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "calibrate_merge workspace");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Carver cv(workspace);
+  CalMergeArgs c;
+  c.obs = cv.take<uint32_t>(16);
+  c.ln = cv.take<float>((size_t)B * ((H + 1) / 2) * ((W + 1) / 2) * K);
+  c.x = x; c.y = y; c.B = B; c.H = H; c.W = W; c.C = C; c.N = N;
+  c.ln_g = p->ln_g; c.ln_b = p->ln_b; c.w = p->reduction.codes; c.sw = p->reduction.scale;
+  g_launches = 0;
+  if (!launch_calibrate_merge(c, st)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "calibrate_merge: unsupported dim");
+  ctx->launches = g_launches;
+  mixaq_status s = check_cuda(ctx, "calibrate_merge");
+  if (s != MIXAQ_OK) return s;
+  return read_ranges(ctx, c.obs, 1, range, st);
+}
+
+mixaq_status mixaq_aq_from_range(float lo, float hi, int bits, mixaq_aq* out) {
+  if (!out || !bits_ok(bits) || !(hi > lo)) return MIXAQ_INVALID_ARG;
+  const int qmax = (1 << bits) - 1;
+  out->bits = bits;
+  out->scale = (float)(((double)hi - (double)lo) / (double)qmax);
+  out->inv_scale = 1.0f / out->scale;
+  double z = std::nearbyint(-(double)lo / (double)out->scale);
+  out->zero_point = (int)std::fmin(std::fmax(z, 0.0), (double)qmax);
   return MIXAQ_OK;
 }
 

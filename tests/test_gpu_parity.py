@@ -382,24 +382,6 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(orc, mq):
         c.close()
 
 
-def test_calibration_on_the_gpu_feeds_the_quantized_forward(orc, mq, ctx):
-    """Min/max calibration run with CUDA tensors, then the library's quantized forward with those quantizers against
-    the oracle with the same quantizers."""
-    from paper_2507_19131_b200 import calibrate
-    wl = synth.tiny_backbone(ratio=0.4)
-    cal = calibrate.calibrate_backbone(wl.backbone, wl.x, device="cuda")
-    ref = calibrate.calibrate_backbone(wl.backbone, wl.x, device="cpu")
-    for a, b in zip(cal.blocks, ref.blocks):
-        for site in calibrate.SITES:
-            assert getattr(a.hi, site).scale == pytest.approx(getattr(b.hi, site).scale, rel=1e-3)
-    want = orc.backbone_forward(cal, wl.x, wl.low_ratios)
-    dbb = mq.DeviceBackbone(ctx, cal, wl.B, wl.H, wl.W)
-    got = mq.backbone_forward(ctx, dbb, dev(wl.x), wl.low_ratios)
-    torch.cuda.synchronize()
-    for g, w in zip(got, want):
-        assert np.array_equal(g.cpu().numpy(), w)
-
-
 def test_mma_issue_rate_microbenchmark(mq, ctx):
     """The library's own tensor-core loop: kind::i8 reaches petaops; kind::f8f6f4 (the path of the 4/6-bit operand
     formats in 8-bit containers) is not faster; kind::mxf4 (block-scaled E2M1, the one narrower path with a higher

@@ -104,7 +104,9 @@ def test_stage_shared_energy_map_is_used_when_given(orc):
 # A textbook Swin block on the un-windowed map, binary64, written from global coordinates: token i attends
 # token j iff both fall into the same window of the cyclically shifted padded frame and the same mask region.
 # ------------------------------------------------------------------------------------------------
-def textbook_block(blk, br, x):
+def textbook_block(blk, br, x, sites=None):
+    """sites (optional dict): filled with (min, max) of what each quantizer site would see, over ALL tokens of the
+    padded map (pad tokens pass through the layers like any token; only the final crop drops them)."""
     B, H, W, C = x.shape
     ws, s, nh = blk.window, blk.shift, blk.heads
     d = C // nh
@@ -117,6 +119,11 @@ def textbook_block(blk, br, x):
 
     def lin(v, L, bias):
         return v @ (L.codes.astype(np.float64) * L.scale.astype(np.float64)[:, None]).T + bias
+
+    def see(name, t):
+        if sites is not None:
+            lo, hi = sites.get(name, (np.inf, -np.inf))
+            sites[name] = (min(lo, float(t.min())), max(hi, float(t.max())))
 
     # coordinates of every padded-frame token in the shifted frame
     yy, xx = np.mgrid[0:Hp, 0:Wp]
@@ -134,10 +141,14 @@ def textbook_block(blk, br, x):
     ridx = (ti[:, None] - ti[None, :] + ws - 1) * (2 * ws - 1) + (tj[:, None] - tj[None, :] + ws - 1)
     out = np.empty_like(x, dtype=np.float64)
     for b in range(B):
-        xb = x[b].astype(np.float64)
+        xb = np.zeros((Hp, Wp, C))
+        xb[:H, :W] = x[b].astype(np.float64)
         n1 = np.zeros((Hp, Wp, C))
-        n1[:H, :W] = ln(xb, br.ln1_g, br.ln1_b)                         # pad tokens are zero AFTER the norm
+        n1[:H, :W] = ln(xb[:H, :W], br.ln1_g, br.ln1_b)                 # pad tokens are zero AFTER the norm
+        see("qkv_in", n1)
         qkv = lin(n1.reshape(-1, C), blk.qkv, br.b_qkv)
+        for i, name in enumerate(("q", "k", "v")):
+            see(name, qkv[:, i * C:(i + 1) * C])
         att = np.zeros((Hp * Wp, C))
         for h in range(nh):
             q, k, v = (qkv[:, i * C + h * d:i * C + (h + 1) * d] for i in range(3))
@@ -146,11 +157,14 @@ def textbook_block(blk, br, x):
             p = np.exp(lg - lg.max(-1, keepdims=True))
             p /= p.sum(-1, keepdims=True)
             att[:, h * d:(h + 1) * d] = p @ v
-        proj = lin(att, blk.proj, br.b_proj).reshape(Hp, Wp, C)[:H, :W]
-        x1 = xb + proj
-        hid = lin(ln(x1, br.ln2_g, br.ln2_b), blk.fc1, br.b_fc1)
+        see("proj_in", att)
+        x1 = xb + lin(att, blk.proj, br.b_proj).reshape(Hp, Wp, C)      # a pad token's residual input is zero
+        n2 = ln(x1, br.ln2_g, br.ln2_b)
+        see("fc1_in", n2)
+        hid = lin(n2, blk.fc1, br.b_fc1)
         hid = 0.5 * hid * (1 + erf(hid / math.sqrt(2)))
-        out[b] = x1 + lin(hid, blk.fc2, br.b_fc2)
+        see("fc2_in", hid)
+        out[b] = (x1 + lin(hid, blk.fc2, br.b_fc2))[:H, :W]
     return out
 
 
@@ -165,6 +179,34 @@ def test_fp_mode_equals_textbook_swin_block(orc, H, W, shift, dim, heads):
     blk.lo = copy.deepcopy(blk.hi)
     got2 = orc.block_forward(blk, x, 0.4, quant=False).y
     assert np.array_equal(got2, got)
+
+
+@pytest.mark.parametrize("H,W,shift,dim,heads", [(10, 12, 3, 32, 1), (14, 14, 0, 64, 2), (8, 9, 3, 32, 1)])
+def test_calibration_observer_ranges_equal_the_textbook_blocks(orc, H, W, shift, dim, heads):
+    """Section 4.3: the ranges come from the floating-point block on the full feature map.  The oracle's observer
+    against the min / max of the same seven tensors of the textbook block (binary64, un-windowed map)."""
+    blk = small_block(seed=H + 7 * shift, dim=dim, heads=heads, shift=shift, share_bias=False)
+    x = small_input(19, 2, H, W, dim)
+    for name in ("hi", "lo"):
+        br = getattr(blk, name)
+        y, got = orc.block_observe_fp(blk, name, x)
+        sites = {}
+        want_y = textbook_block(blk, br, x, sites)
+        assert np.abs(y - want_y).max() < 2e-4 * max(1.0, np.abs(want_y).max())
+        assert np.array_equal(y, orc.uniform_block_forward(blk, name, x, quant=False))
+        for site in orc.SITES:
+            span = sites[site][1] - sites[site][0]
+            assert abs(got[site][0] - sites[site][0]) < 1e-4 * span and abs(got[site][1] - sites[site][1]) < 1e-4 * span, site
+    m = synth.make_merge(np.random.default_rng(23), dim, 8, 8)
+    ym, (lo, hi) = orc.merge_observe_fp(m, x)
+    assert np.array_equal(ym, orc.merge_forward(m, x, quant=False))
+    B = x.shape[0]
+    xp = np.zeros((B, H + H % 2, W + W % 2, dim), np.float64)
+    xp[:, :H, :W] = x
+    cat = np.concatenate([xp[:, 0::2, 0::2], xp[:, 1::2, 0::2], xp[:, 0::2, 1::2], xp[:, 1::2, 1::2]], -1)
+    mu = cat.mean(-1, keepdims=True)
+    n = (cat - mu) / np.sqrt(((cat - mu) ** 2).mean(-1, keepdims=True) + 1e-5) * m.ln_g + m.ln_b
+    assert abs(lo - n.min()) < 1e-4 and abs(hi - n.max()) < 1e-4
 
 
 # ------------------------------------------------------------------------------------------------
