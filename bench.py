@@ -209,9 +209,6 @@ def run_ours(args):
         outs_host = [torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in dbb.outs]
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
 
-        # tile widths of this workload's GEMM shapes, timed once outside the timed region (exact: widths do not change results)
-        tuned = mq.backbone_autotune(ctx, dbb, x_dev, wl.low_ratios, wl.prune_ratios, rounds=3)
-
         def step():
             if e2e:
                 x_dev.copy_(x_host, non_blocking=True)
@@ -238,7 +235,7 @@ def run_ours(args):
         launches = ctx.launch_count()
         h2d = x_host.numel() * 4 if e2e else 0
         d2h = sum(h.numel() * 4 for h in outs_host) if e2e else 0
-        return dict(ms=ms, wall=wall, clocks=clocks, launches=launches, h2d=h2d, d2h=d2h, wl=wl, dbb=dbb, x_dev=x_dev, tuned=tuned)
+        return dict(ms=ms, wall=wall, clocks=clocks, launches=launches, h2d=h2d, d2h=d2h, wl=wl, dbb=dbb, x_dev=x_dev)
 
     def time_e2e(ratio, steps, warm):
         wl = workload(ratio)
@@ -449,7 +446,6 @@ def run_ours(args):
                    "act_bits_high_low": [bbm.blocks[0].hi.bits, bbm.blocks[0].lo.bits], "low_ratio": args.ratio,
                    "prune_ratio": (main["wl"].prune_ratios or [0.0])[0],
                    "l2": f"flushed between timed iterations ({L2_FLUSH_BYTES >> 20} MiB write)",
-                   "gemm_tile_widths": "timed per GEMM shape before the timed region (mixaq_backbone_autotune, 3 rounds; %d shapes)" % main["tuned"],
                    "parallelism": "replicas only (one image per GPU, no collective)"},
         "clocks": main["clocks"],
         "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],

@@ -240,18 +240,6 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
                                     const float* low_ratio_per_pair, const float* prune_ratio_per_pair /* nullable */,
                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Tile-width tuning of the integer GEMMs (the paper has no counterpart: a property of this implementation).  Takes the
- * arguments of mixaq_backbone_forward and runs that forward 8 x `rounds` times: once per candidate tile width (32 ... 256
- * columns) and round, with CUDA events around every GEMM launch; for every GEMM shape that occurs (epilogue, rows of the
- * two branches, N, K, activation bits) the fastest width is remembered in the context and used by every later block,
- * merge and backbone call that launches the same shape.  Results do not depend on the tile width (integer accumulation
- * is exact).  Synchronises the stream; drops the context's captured graphs.  Untuned shapes keep the built-in choice. */
-mixaq_status mixaq_backbone_autotune(mixaq_ctx* ctx, const mixaq_backbone_params* p, const float* x0,
-                                     float* const* stage_out, int B, int H0, int W0,
-                                     const float* low_ratio_per_pair, const float* prune_ratio_per_pair /* nullable */,
-                                     void* workspace, size_t workspace_bytes, void* cuda_stream, int rounds);
-int          mixaq_tuned_shape_count(const mixaq_ctx* ctx);
-
 /* mixaq_backbone_forward replays a CUDA graph when it is called again with exactly the same arguments (same
  * parameter structs byte for byte, pointers, sizes, ratios, workspace and stream): the first such call captures the
  * launches on `cuda_stream`, later calls cost one graph launch on the host.  The data behind the pointers may

@@ -24,7 +24,7 @@ EXPORTS = [
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
     "mixaq_norm_forward", "mixaq_profile_end_records", "mixaq_calibrate_block_workspace_bytes", "mixaq_calibrate_block",
-    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection", "mixaq_backbone_autotune", "mixaq_tuned_shape_count",
+    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -451,18 +451,6 @@ def calibrate_merge(ctx: Context, merge_struct: MergeS, x: torch.Tensor):
     ctx.check(lib().mixaq_calibrate_merge(ctx.h, C.byref(merge_struct), _ptr(x), _ptr(y), B, H, W, C.byref(r), _ptr(ws),
                                           C.c_size_t(ws.numel()), _stream_ptr()), "calibrate_merge")
     return y, (float(r.lo), float(r.hi))
-
-
-def backbone_autotune(ctx: Context, dbb: "DeviceBackbone", x0: torch.Tensor, low_ratios, prune_ratios=None, rounds: int = 3) -> int:
-    """mixaq_backbone_autotune: times every GEMM shape of this forward at every tile width and keeps the fastest per
-    shape in the context.  Returns the number of tuned shapes the context holds."""
-    lr = (C.c_float * dbb.npairs)(*[float(r) for r in low_ratios][:dbb.npairs])
-    pr = None
-    if prune_ratios is not None:
-        pr = (C.c_float * dbb.npairs)(*[float(r) for r in prune_ratios][:dbb.npairs])
-    ctx.check(lib().mixaq_backbone_autotune(ctx.h, C.byref(dbb.s), _ptr(x0), dbb.out_ptrs, dbb.B, dbb.H0, dbb.W0, lr, pr,
-                                            _ptr(dbb.ws), C.c_size_t(dbb.ws.numel()), _stream_ptr(), rounds), "backbone_autotune")
-    return lib().mixaq_tuned_shape_count(ctx.h)
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

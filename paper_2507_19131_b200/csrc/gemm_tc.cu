@@ -447,7 +447,7 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   if (g.N % 32 || g.K % UMMA_K) return false;
   const int sms = num_sms();
   p.tiles_m0 = t0;
-  p.BN = (g.bn > 0 && g.bn <= MAX_BN && g.bn % 32 == 0 && g.N % g.bn == 0) ? g.bn : pick_bn(g.N, t0 + t1, sms);
+  p.BN = pick_bn(g.N, t0 + t1, sms);
   if (p.BN == 0) return false;
   p.n_tiles = g.N / p.BN;
   p.total_tiles = (t0 + t1) * p.n_tiles;
@@ -609,10 +609,6 @@ bool gemm_init() {
   ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
   ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
   return ok;
-}
-
-int gemm_default_bn(int N, int M0, int M1) {
-  return pick_bn(N, (M0 + BM - 1) / BM + (M1 + BM - 1) / BM, num_sms());
 }
 
 bool launch_gemm(const GemmArgs& g, cudaStream_t st) {

@@ -77,10 +77,8 @@ struct GemmArgs {
   int N, K, C;               // C: channels per q/k/v section (EPI_QKV)
   int mode;
   int* status;           // device status word (raised when a bounded wait runs out)
-  int bn;                // tile width to use (a multiple of 32 that divides N, at most 256); 0: the launcher's own choice
   GemmBranch br[2];
 };
-int gemm_default_bn(int N, int M0, int M1);   // the launcher's own choice of tile width
 bool launch_gemm(const GemmArgs& g, cudaStream_t st);
 void launch_wait_probe(int* status, cudaStream_t st);   // self-test of the bounded wait (it must run out)
 // tensor-core issue-rate microbenchmark (kind 0: i8, 1: f8f6f4/E4M3); ns per SM into ns_out; returns the grid size

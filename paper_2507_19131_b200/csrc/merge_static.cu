@@ -111,7 +111,7 @@ extern "C" mixaq_status mixaq_merge_forward_static(mixaq_ctx* ctx, const mixaq_m
   int32_t* zc = reinterpret_cast<int32_t*>(static_cast<char*>(p->prepared) + round256((size_t)N * 4));
   GemmArgs ga;
   ga.status = ctx_status_word(ctx);
-  ga.w = p->reduction.codes; ga.N = N; ga.K = K; ga.C = N; ga.mode = EPI_MERGE; ga.bn = 0;
+  ga.w = p->reduction.codes; ga.N = N; ga.K = K; ga.C = N; ga.mode = EPI_MERGE;
   for (int i = 0; i < 2; ++i) {
     memset(&ga.br[i], 0, sizeof(GemmBranch));
     ga.br[i].a_bits = bits; ga.br[i].mult = mult; ga.br[i].zc = zc;

@@ -3,11 +3,9 @@
 // Nothing here computes: every step of the path runs in the kernels.
 #include "../../include/mixaq.h"
 #include "kernels.h"
-#include <array>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
-#include <map>
 #include <new>
 #include <string>
 #include <vector>
@@ -21,9 +19,6 @@ thread_local int g_launches = 0;
 using namespace mixaq;
 
 struct ProfRec { int cat; cudaEvent_t e0, e1; };
-// A GEMM launch as the tile-width tuner sees it: epilogue mode, rows of the two branches, N, K, activation bits.
-typedef std::array<int, 7> GemmShape;
-struct TuneSample { GemmShape shape; int bn; size_t prof_index; };
 // One captured backbone forward: the exact bytes of every argument that shaped it, and the instantiated graph.
 struct GraphEntry { std::string key; cudaGraphExec_t exec; int launches; };
 struct mixaq_ctx {
@@ -35,10 +30,6 @@ struct mixaq_ctx {
   bool graph_cache;                    // replay backbone forwards as CUDA graphs (see mixaq_set_graph_cache)
   bool reverse_selection;              // backbone: worst-case selection order (Table 4) in every block
   bool allow_elevation;                // backbone: every pair uses its own ratios even if an earlier pair of the stage had larger ones
-  std::map<GemmShape, int> bn_table;   // tuned tile widths (mixaq_backbone_autotune)
-  int tune_force_bn;                   // > 0 while the tuner sweeps: try this width wherever it divides N
-  bool tune_logging;
-  std::vector<TuneSample> tune_log;    // GEMM launches of the sweep in issue order
   std::vector<GraphEntry> graphs;
   std::vector<ProfRec> prof;          // event pairs recorded since mixaq_profile_begin
   std::vector<cudaEvent_t> pool;      // events ready for reuse
@@ -224,20 +215,6 @@ SelectArgs make_select_args(const SelWs& sel, const int32_t* energy, int B, int 
   return sa;
 }
 
-// Tile width of a GEMM launch: the tuned one when the shape was tuned, the sweep's candidate while tuning, else 0
-// (the launcher's own choice).  While the tuner logs, the launch is recorded with the profiling record it will get.
-int choose_bn(mixaq_ctx* ctx, const GemmArgs& ga) {
-  const GemmShape shape = {ga.mode, ga.br[0].M, ga.br[1].M, ga.N, ga.K, ga.br[0].a_bits, ga.br[1].a_bits};
-  int bn = 0;
-  if (ctx->tune_force_bn > 0) { if (ga.N % ctx->tune_force_bn == 0) bn = ctx->tune_force_bn; }
-  else { auto it = ctx->bn_table.find(shape); if (it != ctx->bn_table.end()) bn = it->second; }
-  if (ctx->tune_logging) {
-    const int used = bn > 0 ? bn : gemm_default_bn(ga.N, ga.br[0].M, ga.br[1].M);
-    ctx->tune_log.push_back({shape, used, ctx->prof.size()});      // the next profiling record is this launch's
-  }
-  return bn;
-}
-
 void fill_gemm_branch(GemmBranch& g, const uint8_t* a, int M, int a_bits, const float* mult, const int32_t* zc,
                       const float* bias) {
   memset(&g, 0, sizeof(g));
@@ -267,7 +244,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false; c->tune_force_bn = 0; c->tune_logging = false;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
       !gemm_init()) {
     cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
@@ -500,7 +477,6 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.qkv[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->qkv_acc : nullptr;
   }
-  ga.bn = choose_bn(ctx, ga);
   { PROF(PC_QKV); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 4. window attention
@@ -526,7 +502,6 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = sel.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->proj_acc : nullptr;
   }
-  ga.bn = choose_bn(ctx, ga);
   { PROF(PC_PROJ); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 6. LN2 + quantize + pack
@@ -543,7 +518,6 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     ga.br[i].q0 = to_aq(brp[i]->fc2_in); ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.f2[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc1_acc : nullptr;
   }
-  ga.bn = choose_bn(ctx, ga);
   { PROF(PC_FC1); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 8. fc2 GEMM + residual + scatter (reverse shift, crop)
@@ -553,7 +527,6 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = sel.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc2_acc : nullptr;
   }
-  ga.bn = choose_bn(ctx, ga);
   { PROF(PC_FC2); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
 
   // 9. pruned windows are forwarded unchanged
@@ -619,7 +592,6 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
   fill_gemm_branch(ga.br[0], (const uint8_t*)workspace, M, p->in.bits, mult, zc, nullptr);
   ga.br[0].out_f = y;
   fill_gemm_branch(ga.br[1], nullptr, 0, p->in.bits, mult, zc, nullptr);
-  ga.bn = choose_bn(ctx, ga);
   { PROF(PC_MERGE_GEMM); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
   ctx->launches = g_launches;
   return check_cuda(ctx, "merge_forward");
@@ -860,59 +832,6 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
 }
 
 // -------------------------------------------------------------------------------------------------
-// Tile-width tuning: every GEMM shape of this forward is timed at every tile width that divides its N (CUDA events
-// around each launch, direct launches, minimum over the rounds); the fastest width per shape is kept in the context.
-mixaq_status mixaq_backbone_autotune(mixaq_ctx* ctx, const mixaq_backbone_params* p, const float* x0,
-                                     float* const* stage_out, int B, int H0, int W0,
-                                     const float* low_ratio_per_pair, const float* prune_ratio_per_pair,
-                                     void* workspace, size_t workspace_bytes, void* cuda_stream, int rounds) {
-  if (!ctx) return MIXAQ_INVALID_ARG;
-  if (rounds <= 0 || ctx->profiling) return fail(ctx, MIXAQ_INVALID_ARG, "autotune: rounds must be positive and profiling off");
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  static const int kWidths[] = {32, 64, 96, 128, 160, 192, 224, 256};
-  std::map<GemmShape, std::map<int, float>> best;          // shape -> width -> fastest time seen
-  mixaq_status result = MIXAQ_OK;
-  for (int wi = 0; wi < 8 && result == MIXAQ_OK; ++wi) {
-    ctx->tune_force_bn = kWidths[wi];
-    for (int r = 0; r < rounds && result == MIXAQ_OK; ++r) {
-      ctx->tune_log.clear();
-      mixaq_profile_begin(ctx);
-      ctx->tune_logging = true;
-      result = mixaq_backbone_forward(ctx, p, x0, stage_out, B, H0, W0, low_ratio_per_pair, prune_ratio_per_pair,
-                                      workspace, workspace_bytes, cuda_stream);
-      ctx->tune_logging = false;
-      ctx->profiling = false;
-      if (cudaStreamSynchronize(st) != cudaSuccess) result = check_cuda(ctx, "autotune") == MIXAQ_OK ? MIXAQ_CUDA_ERROR : MIXAQ_CUDA_ERROR;
-      if (result == MIXAQ_OK)
-        for (const TuneSample& smp : ctx->tune_log) {
-          if (smp.prof_index >= ctx->prof.size()) continue;
-          float ms = 0.f;
-          if (cudaEventElapsedTime(&ms, ctx->prof[smp.prof_index].e0, ctx->prof[smp.prof_index].e1) != cudaSuccess) { cudaGetLastError(); continue; }
-          auto& slot = best[smp.shape];
-          auto it = slot.find(smp.bn);
-          if (it == slot.end() || ms < it->second) slot[smp.bn] = ms;
-        }
-      for (auto& rec : ctx->prof) { ctx->pool.push_back(rec.e0); ctx->pool.push_back(rec.e1); }
-      ctx->prof.clear();
-    }
-  }
-  ctx->tune_force_bn = 0;
-  ctx->tune_log.clear();
-  if (result != MIXAQ_OK) return result;
-  for (auto& kv : best) {
-    int bn = 0; float t = 0.f;
-    for (auto& wt : kv.second) if (!bn || wt.second < t) { bn = wt.first; t = wt.second; }
-    if (bn) ctx->bn_table[kv.first] = bn;
-  }
-  // forwards captured before the tuning used other widths
-  for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
-  ctx->graphs.clear();
-  return MIXAQ_OK;
-}
-
-int mixaq_tuned_shape_count(const mixaq_ctx* ctx) { return ctx ? (int)ctx->bn_table.size() : 0; }
-
-// -------------------------------------------------------------------------------------------------
 // stem and output norms
 namespace {
 constexpr int EMBED_K = 48, EMBED_KP = 64;     // patch vector, padded to a multiple of 32 codes
@@ -973,7 +892,7 @@ mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, co
   launch_patch_gather(pg, st);
   GemmArgs ga;
   ga.status = ctx->d_status;
-  ga.w = pr.w; ga.N = N; ga.K = EMBED_KP; ga.C = N; ga.mode = EPI_MERGE; ga.bn = 0;      // dequantize only: acc * mult
+  ga.w = pr.w; ga.N = N; ga.K = EMBED_KP; ga.C = N; ga.mode = EPI_MERGE;      // dequantize only: acc * mult
   fill_gemm_branch(ga.br[0], codes, (int)toks, 8, pr.mult, pr.zc, nullptr);
   ga.br[0].out_f = t;
   fill_gemm_branch(ga.br[1], nullptr, 0, 8, pr.mult, pr.zc, nullptr);
