@@ -71,7 +71,8 @@ __device__ __forceinline__ uint32_t squeeze_pairs(uint32_t t) {
   return t;
 }
 
-template <bool SHIFTED>
+// TAPS: the debug taps (softmax output, P codes, P.V accumulators) are compiled in only for calls that ask for them
+template <bool SHIFTED, bool TAPS>
 __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
   __shared__ __align__(16) WarpSmem sm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -216,7 +217,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
 #pragma unroll
         for (int nt = 0; nt < 7; ++nt) {
           const float2 pr = __fmul2_rn(lg[nt], f2(inv));          // the softmax output itself
-          if (br.tap_probs) {
+          if (TAPS && br.tap_probs) {
             const int j0 = 8 * nt + 2 * t;
             float* tp = br.tap_probs + (((long)slot * a.heads + h) * WT + i) * WT;
             if (i < WT && j0 < WT) tp[j0] = pr.x;
@@ -231,7 +232,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
           for (int u = 0; u < 2; ++u) {
             ps += (int)code[u];
             pa[ks][r + 2 * (sub >> 1)] |= code[u] << (8 * (2 * (sub & 1) + u));
-            if (br.tap_p) {
+            if (TAPS && br.tap_p) {
               const int j = 8 * nt + 2 * t + u;
               if (i < WT && j < WT) br.tap_p[(((long)slot * a.heads + h) * WT + i) * WT + j] = (uint8_t)code[u];
             }
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
 #pragma unroll
       for (int ne = 0; ne < 4; ++ne) {
         const int o0 = d[ne][2 * r] - zv * psum[r], o1 = d[ne][2 * r + 1] - zv * psum[r];
-        if (br.tap_pv && r < nrows && i < WT) {
+        if (TAPS && br.tap_pv && r < nrows && i < WT) {
           int* tp = br.tap_pv + (m_base + i) * C + h * HEAD_DIM + 8 * ne + 2 * t;
           tp[0] = o0; tp[1] = o1;
         }
@@ -300,8 +301,14 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   const long problems = (long)(a.br[0].slots + a.br[1].slots) * a.heads;
   if (problems == 0) return;
   const unsigned grid = (unsigned)problems;
-  if (a.shift > 0) k_attention<true><<<grid, ATT_WARPS * 32, 0, st>>>(a);
-  else             k_attention<false><<<grid, ATT_WARPS * 32, 0, st>>>(a);
+  const bool taps = a.br[0].tap_p || a.br[0].tap_pv || a.br[0].tap_probs || a.br[1].tap_p || a.br[1].tap_pv || a.br[1].tap_probs;
+  if (a.shift > 0) {
+    if (taps) k_attention<true, true><<<grid, ATT_WARPS * 32, 0, st>>>(a);
+    else      k_attention<true, false><<<grid, ATT_WARPS * 32, 0, st>>>(a);
+  } else {
+    if (taps) k_attention<false, true><<<grid, ATT_WARPS * 32, 0, st>>>(a);
+    else      k_attention<false, false><<<grid, ATT_WARPS * 32, 0, st>>>(a);
+  }
   ++g_launches;
 }
 
