@@ -37,10 +37,10 @@ __device__ __forceinline__ void tmem_ld_wait(int32_t (&r)[16]) {
 }
 
 // zero-point correction + dequantization of one chunk; lc0 = first column of the chunk in the warp's constants
-template <int MODE>
+template <int MODE, bool TAPS>
 __device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, bool row_ok, int n0, int lc0,
                                           const ColConsts& cc, const int32_t (&acc_raw)[16], float (&v)[16]) {
-  if (br.tap_acc && row_ok) {
+  if (TAPS && br.tap_acc && row_ok) {
 #pragma unroll
     for (int i = 0; i < EPI_NC; ++i) br.tap_acc[m * N + n0 + i] = acc_raw[i] - cc.zc[lc0 + i];
   }
@@ -71,7 +71,7 @@ __device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, b
 // n_tile0: global index of that column; the warp owns the tile's chunks c_first, c_first + c_step, ... < c_total
 // (its constants are stored densely: chunk number j of the warp at local column 16 j);
 // acc_ready(): waits (bounded) for the tile's accumulator, false when the CTA is giving up.
-template <int MODE, class WaitFn>
+template <int MODE, bool TAPS, class WaitFn>
 __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, int C, long row0, int lane, int n_tile0,
                                                    int c_first, int c_step, int c_total, const ColConsts& cc,
                                                    uint32_t taddr_tile, float* stage, WaitFn acc_ready) {
@@ -96,7 +96,7 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
       const int n0 = n_first + ch * col_step;
       float v[EPI_NC];
-      dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
+      dequant16<MODE, TAPS>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
       AQ q = br.q0;
       uint32_t kp = kp0;
       if (MODE == EPI_QKV) { if (n0 >= n_v) { q = br.q2; kp = kp2; } else if (n0 >= n_k) { q = br.q1; kp = kp1; } }
@@ -166,7 +166,7 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
   auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
     const int n0 = n_first + ch * col_step;
     float v[EPI_NC];
-    dequant16<MODE>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
+    dequant16<MODE, TAPS>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
     if (ch + 1 < n_chunks) fetch(ch + 1, res_next);
     // row `lane`, logical 16-byte piece j is stored at piece j ^ ((lane >> 1) & 3): conflict-free both ways
 #pragma unroll

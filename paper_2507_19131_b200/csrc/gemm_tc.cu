@@ -130,7 +130,8 @@ __device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int t) {
   return c;
 }
 
-template <int MODE>
+// TAPS: the accumulator tap is compiled in only for calls that ask for it
+template <int MODE, bool TAPS>
 __global__ void __launch_bounds__(32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
           const __grid_constant__ CUtensorMap tmB, const TcParams p) {
@@ -339,7 +340,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         return true;
       };
-      if (!epilogue_warp_tile<MODE>(br, p.g.N, p.g.C, row0, lane, n_tile0, sub, EPI_SPLIT, c_total, cc, taddr, stage,
+      if (!epilogue_warp_tile<MODE, TAPS>(br, p.g.N, p.g.C, row0, lane, n_tile0, sub, EPI_SPLIT, c_total, cc, taddr, stage,
                                     acc_ready)) break;
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -481,7 +482,10 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles)
   int grid = p.total_tiles < sms ? p.total_tiles : sms;
   if (grid > p.n_tiles && grid < p.total_tiles) grid -= grid % p.n_tiles;
-  k_gemm_tc<MODE><<<grid, 32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), smem, st>>>(mA[0], mA[1], mB, p);
+  if (g.br[0].tap_acc || g.br[1].tap_acc)
+    k_gemm_tc<MODE, true><<<grid, 32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), smem, st>>>(mA[0], mA[1], mB, p);
+  else
+    k_gemm_tc<MODE, false><<<grid, 32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), smem, st>>>(mA[0], mA[1], mB, p);
   ++g_launches;
   return true;
 }
@@ -603,11 +607,16 @@ int launch_mma_peak(int kind, int groups, unsigned long long* ns_out, int* statu
 // opt-in to large dynamic shared memory for every epilogue mode, resolve the tensor-map encoder, read the SM count.
 bool gemm_init() {
   bool ok = encode_fn() != nullptr && num_sms() > 0;
-  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
-  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_QKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_PROJ, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_PROJ, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_FC2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_MERGE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  ok &= cudaFuncSetAttribute(k_gemm_tc<EPI_MERGE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
   return ok;
 }
 
