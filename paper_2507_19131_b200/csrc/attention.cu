@@ -212,8 +212,12 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
         const float s1 = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, 1));
         const float sum = __fadd_rn(s1, __shfl_xor_sync(0xffffffffu, s1, 2));
         const float inv = __fdiv_rn(1.0f, sum);
-        // P codes: clamp(rne(p * pmax), 0, pmax); byte u of A register (ks, r [+2]) is tile 4ks + [2 +] (u>>1), column u&1
-        int ps = 0;
+        // P codes: clamp(rne(p * pmax), 0, pmax); byte u of A register (ks, r [+2]) is tile 4ks + [2 +] (u>>1), column u&1.
+        // The clamp never acts: 0 <= e_j <= sum, so p * pmax lies in [0, pmax * (1 + 2^-22)] and rounds into 0 .. pmax;
+        // it is left out.  The rounded values stay in their "1.5 * 2^23 + code" patterns: the patterns are added into
+        // the A registers shifted into place and the bias they carry is taken out once per register.
+        uint32_t acc_pa[4] = {0u, 0u, 0u, 0u};
+        uint32_t ps_raw = 0u;
 #pragma unroll
         for (int nt = 0; nt < 7; ++nt) {
           const float2 pr = __fmul2_rn(lg[nt], f2(inv));          // the softmax output itself
@@ -223,21 +227,30 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
             if (i < WT && j0 < WT) tp[j0] = pr.x;
             if (i < WT && j0 + 1 < WT) tp[j0 + 1] = pr.y;
           }
-          float2 tq = __fmul2_rn(pr, f2(pmaxf));
-          tq = make_float2(fminf(fmaxf(tq.x, 0.0f), pmaxf), fminf(fmaxf(tq.y, 0.0f), pmaxf));
-          tq = __fadd2_rn(tq, f2(12582912.0f));
-          const uint32_t code[2] = {__float_as_uint(tq.x) - kMagicBits, __float_as_uint(tq.y) - kMagicBits};
+          // two roundings (product, then the add that rounds to an integer).  The products are scalar multiplies: a
+          // packed multiply feeding a packed add gets contracted into one fused operation, which rounds once and
+          // differs at exact .5 ties
+          const float2 tq = __fadd2_rn(make_float2(__fmul_rn(pr.x, pmaxf), __fmul_rn(pr.y, pmaxf)), f2(12582912.0f));
+          const uint32_t pat[2] = {__float_as_uint(tq.x), __float_as_uint(tq.y)};
           const int ks = nt >> 2, sub = nt & 3;
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
-            ps += (int)code[u];
-            pa[ks][r + 2 * (sub >> 1)] |= code[u] << (8 * (2 * (sub & 1) + u));
+            ps_raw += pat[u];
+            acc_pa[2 * ks + (sub >> 1)] += pat[u] << (8 * (2 * (sub & 1) + u));
             if (TAPS && br.tap_p) {
               const int j = 8 * nt + 2 * t + u;
-              if (i < WT && j < WT) br.tap_p[(((long)slot * a.heads + h) * WT + i) * WT + j] = (uint8_t)code[u];
+              if (i < WT && j < WT) br.tap_p[(((long)slot * a.heads + h) * WT + i) * WT + j] = (uint8_t)(pat[u] - kMagicBits);
             }
           }
         }
+        // register (ks, half): four patterns (three for ks = 1, half = 1: tiles 4..6 only); the low byte of a pattern's
+        // bias 0x4B400000 is zero, so shifted into a byte lane it only reaches higher bytes, which the sum drops
+        // beyond bit 31: bias of a register = sum over its lanes of (0x4B400000 << 8 lane) mod 2^32
+        constexpr uint32_t kBias4 = kMagicBits + (kMagicBits << 8) + (kMagicBits << 16) + (kMagicBits << 24);
+        constexpr uint32_t kBias2 = kMagicBits + (kMagicBits << 8);
+        pa[0][r] = acc_pa[0] - kBias4;  pa[0][r + 2] = acc_pa[1] - kBias4;
+        pa[1][r] = acc_pa[2] - kBias4;  pa[1][r + 2] = acc_pa[3] - kBias2;
+        int ps = (int)(ps_raw - 14u * kMagicBits);
         ps += __shfl_xor_sync(0xffffffffu, ps, 1);
         ps += __shfl_xor_sync(0xffffffffu, ps, 2);
         psum[r] = ps;

@@ -21,6 +21,10 @@ struct AQ {                   // activation quantizer in kernel-friendly form
 // bit-identical to the scalar function applied to .x and .y; one packed instruction takes one issue slot where two
 // scalar ones take two, which is what the issue-bound epilogues need.  a - b is written fma(b, -1, a): b * -1 is
 // exact, so the single rounding is that of the subtraction.
+// Caution: unlike the scalar _rn intrinsics, a packed multiply whose result feeds a packed add directly has been seen
+// contracted into one packed fused multiply-add (one rounding instead of two, even with --fmad=false).  Wherever the
+// contract wants the product rounded before the add, an instruction must sit between the two (a clamp) or the product
+// must be formed by scalar multiplies (an empty asm statement between them does not help).
 __device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
 __device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, f2(-1.0f), a); }
 
