@@ -3,6 +3,7 @@
 // Two LayerNorm kernels with the same summation tree: one warp per row (lane l holds channels l, l+32, l+64, ...,
 // every load a full 128-byte line) and, for large batches of narrow rows, 4 or 8 lanes per row with vector loads.
 #include "kernels.h"
+#include <type_traits>
 
 namespace mixaq {
 
@@ -118,42 +119,56 @@ __global__ void __launch_bounds__(256, 4) k_ln_quant_g(LnBranch hi, LnBranch lo,
   const float var = __fdiv_rn(reduce32(p), (float)C);
   const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, 1e-5f)));
   if (m >= M) return;
-  uint8_t* out = br.out + (long)m * (C * bits / 8) + (P * j) * bits / 8;
-  const uint32_t kpack = pack_const(q.zp, bits);
-  const uint32_t zpat = quant_magic(0.0f, q);      // pad token: zero after the normalisation
-  const int per = 32 / bits;                       // codes per 32-bit word
+  // the normalisation, the quantizer and the packing with the bit width as a compile-time constant (a CTA works for
+  // one branch, so the switch is uniform)
+  auto finish = [&](auto bits_tag) {
+    constexpr int BITS = decltype(bits_tag)::value;
+    constexpr int PER = 32 / BITS;                     // codes per 32-bit word
+    uint8_t* out = br.out + (long)m * (C * BITS / 8) + (P * j) * BITS / 8;
+    const uint32_t kpack = pack_const(q.zp, BITS);
+    // a pad token is zero after the normalisation: all its codes are the code of zero
+    uint32_t zw0 = kpack, zw1 = kpack;
+    {
+      const uint32_t zpat = quant_magic(0.0f, q);
 #pragma unroll
-  for (int i = 0; i < NG; ++i) {
-    uint32_t w0 = kpack, w1 = kpack;
+      for (int k = 0; k < P; ++k) { if (k < PER) zw0 += zpat << (BITS * k); else zw1 += zpat << (BITS * (k - PER)); }
+    }
 #pragma unroll
-    for (int v4 = 0; v4 < P / 4; ++v4) {
-      const float4 g4 = __ldg(reinterpret_cast<const float4*>(br.gamma + 32 * i + P * j) + v4);
-      const float4 b4 = __ldg(reinterpret_cast<const float4*>(br.beta + 32 * i + P * j) + v4);
-      const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
+    for (int i = 0; i < NG; ++i) {
+      uint32_t w0 = kpack, w1 = kpack;
 #pragma unroll
-      for (int e = 0; e < 4; e += 2) {
-        const int k = 4 * v4 + e;
-        // y = fma((x - mean) * rstd, gamma, beta) on two channels, then their magic patterns
-        const float2 d = __fmul2_rn(sub2(make_float2(x[i][k], x[i][k + 1]), f2(mean)), f2(rstd));
-        const float2 y = __ffma2_rn(d, make_float2(gg[e], gg[e + 1]), make_float2(bb[e], bb[e + 1]));
-        uint32_t pat[2];
-        quant_magic2(y, q.inv_scale, -q.zpf, q.qmaxf - q.zpf, pat[0], pat[1]);
+      for (int v4 = 0; v4 < P / 4; ++v4) {
+        const float4 g4 = __ldg(reinterpret_cast<const float4*>(br.gamma + 32 * i + P * j) + v4);
+        const float4 b4 = __ldg(reinterpret_cast<const float4*>(br.beta + 32 * i + P * j) + v4);
+        const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const uint32_t pt = srow < 0 ? zpat : pat[u];
-          if (k + u < per) w0 += pt << (bits * (k + u));
-          else             w1 += pt << (bits * (k + u - per));
+        for (int e = 0; e < 4; e += 2) {
+          const int k = 4 * v4 + e;
+          // y = fma((x - mean) * rstd, gamma, beta) on two channels, then their magic patterns
+          const float2 d = __fmul2_rn(sub2(make_float2(x[i][k], x[i][k + 1]), f2(mean)), f2(rstd));
+          const float2 y = __ffma2_rn(d, make_float2(gg[e], gg[e + 1]), make_float2(bb[e], bb[e + 1]));
+          uint32_t pat[2];
+          quant_magic2(y, q.inv_scale, -q.zpf, q.qmaxf - q.zpf, pat[0], pat[1]);
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            if (k + u < PER) w0 += pat[u] << (BITS * (k + u));
+            else             w1 += pat[u] << (BITS * (k + u - PER));
+          }
         }
       }
+      if (srow < 0) { w0 = zw0; w1 = zw1; }
+      // P codes of BITS bits: P*BITS/8 whole bytes (the launcher only picks G with P*BITS >= 8)
+      uint8_t* dst = out + 32 * i * BITS / 8;
+      constexpr int NBYTES = P * BITS / 8;
+      if (NBYTES == 8) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
+      else if (NBYTES == 4) *reinterpret_cast<uint32_t*>(dst) = w0;
+      else if (NBYTES == 2) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)w0;
+      else *dst = (uint8_t)w0;
     }
-    // P codes of `bits` bits: P*bits/8 whole bytes (the launcher only picks G with P*bits >= 8)
-    uint8_t* dst = out + 32 * i * bits / 8;
-    const int nbytes = P * bits / 8;
-    if (nbytes == 8) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
-    else if (nbytes == 4) *reinterpret_cast<uint32_t*>(dst) = w0;
-    else if (nbytes == 2) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)w0;
-    else *dst = (uint8_t)w0;
-  }
+  };
+  if (bits == 8) finish(std::integral_constant<int, 8>{});
+  else if (bits == 4) finish(std::integral_constant<int, 4>{});
+  else finish(std::integral_constant<int, 2>{});
 }
 
 // patch merging: token (b, y2, x2) of the output gathers (2y2+dy, 2x2+dx) for (dy,dx) = (0,0),(1,0),(0,1),(1,1)
