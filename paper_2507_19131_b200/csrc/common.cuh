@@ -83,9 +83,9 @@ __device__ __forceinline__ uint32_t quant_code(float x, const AQ& q) {
 // Additive constant that turns sum_i pattern_i << (bits*i) into the packed word of the codes (the per-code
 // offsets zp - 0x4B400000 are folded into one 32-bit constant; every code fits its field, so nothing carries).
 __device__ __forceinline__ uint32_t pack_const(int zp, int bits) {
-  uint32_t k = (uint32_t)zp - kMagicBits, r = 0;
-  for (int sh = 0; sh < 32; sh += bits) r += k << sh;
-  return r;
+  // sum over the fields of k << shift = k * (sum of 2^shift) modulo 2^32
+  const uint32_t k = (uint32_t)zp - kMagicBits;
+  return k * (bits == 8 ? 0x01010101u : (bits == 4 ? 0x11111111u : 0x55555555u));
 }
 // NC (16 or 32) consecutive codes of one row, given as magic patterns, packed and stored with one or two vector
 // stores (dst is NC*BITS/8-byte aligned).

@@ -310,8 +310,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     float* c_bias = c_mult + EPI_WARP_COLS;
     const int c_total = p.BN / EPI_NC;                         // BN is a multiple of 32
     int lt = 0, consts_key = -1;
+    // the tile walk without a division per tile: (row tile, column tile) advance by gridDim.x tiles at a time
+    const int step_m = (int)gridDim.x / p.n_tiles, step_n = (int)gridDim.x % p.n_tiles;
+    int w_mt = (int)blockIdx.x / p.n_tiles, w_nt = (int)blockIdx.x % p.n_tiles;
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++lt) {
-      const TileCoord tc = decode_tile(p, t);
+      TileCoord tc;
+      tc.nt = w_nt; tc.mt = w_mt; tc.is_hi = w_mt < p.tiles_m0;
+      if (!tc.is_hi) tc.mt -= p.tiles_m0;
+      w_mt += step_m; w_nt += step_n;
+      if (w_nt >= p.n_tiles) { w_nt -= p.n_tiles; ++w_mt; }
       const GemmBranch& br = tc.is_hi ? p.g.br[0] : p.g.br[1];
       const int a = lt & 1;
       const int n_tile0 = tc.nt * p.BN;
