@@ -36,6 +36,15 @@ __device__ __forceinline__ void tmem_ld_wait(int32_t (&r)[16]) {
       :: "memory");
 }
 
+// asynchronous 16-byte copy global -> shared (no register staging); groups complete in order
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int RES_SLOTS = 4;                           // residual chunks a warp keeps in flight (32 x 16 floats each)
+
 // zero-point correction + dequantization of one chunk; lc0 = first column of the chunk in the warp's constants
 template <int MODE, bool TAPS>
 __device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, bool row_ok, int n0, int lc0,
@@ -74,7 +83,8 @@ __device__ __forceinline__ void dequant16(const GemmBranch& br, int N, long m, b
 template <int MODE, bool TAPS, class WaitFn>
 __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, int C, long row0, int lane, int n_tile0,
                                                    int c_first, int c_step, int c_total, const ColConsts& cc,
-                                                   uint32_t taddr_tile, float* stage, WaitFn acc_ready) {
+                                                   uint32_t taddr_tile, float* stage, WaitFn acc_ready,
+                                                   float* res_ring = nullptr /* per warp: RES_SLOTS x 32 x 16 floats */) {
   const long m = row0 + lane;
   const bool row_ok = m < br.M;
   const int n_chunks = c_first < c_total ? (c_total - c_first + c_step - 1) / c_step : 0;
@@ -132,8 +142,7 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
 
   // ---- binary32 outputs (proj: x1 = x_window + out; fc2: y = x1 + out scattered to the token's own position;
   //      merge: out).  Each chunk is transposed through shared memory so that global accesses are 64-byte runs
-  //      (4 lanes per row, 8 rows per instruction).  The residual of chunk ch+1 is fetched while chunk ch is
-  //      computed; the residual of chunk 0 is fetched before the accumulator is even complete. ----
+  //      (4 lanes per row, 8 rows per instruction). ----
   const int cj = lane & 3, rsub = lane >> 2;
   long src_mine = -1;
   if (MODE != EPI_MERGE && row_ok) src_mine = br.rowsrc[m];
@@ -153,44 +162,59 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     res_ptr[i] = (MODE != EPI_MERGE && res_row >= 0) ? br.res + res_row + n_first + 4 * cj : nullptr;
     dst_ptr[i] = dst_row >= 0 ? br.out_f + dst_row + n_first + 4 * cj : nullptr;
   }
-  float4 res[4], res_next[4];
-  auto fetch = [&](int ch, float4 (&dst)[4]) {
+  // The residual rows come into shared memory by asynchronous copies, RES_SLOTS chunks ahead of their use: the copies
+  // of a whole tile are in flight while the accumulator is still being computed, and they cost no registers.
+  // Slot ch % RES_SLOTS holds chunk ch in the layout of the transposition tile (row r, 16-byte piece j at piece
+  // j ^ ((r >> 1) & 3)).  One commit group per chunk, also when there is nothing left to fetch, so that "all but the
+  // newest RES_SLOTS - 1 groups are complete" always covers the chunk about to be used.
+  auto fetch = [&](int ch) {
+    if (MODE != EPI_MERGE && ch < n_chunks) {
+      float* slot = res_ring + (ch % RES_SLOTS) * EPI_STAGE_FLOATS;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);       // a pad token's residual input is zero
-      if (res_ptr[i]) dst[i] = __ldg(reinterpret_cast<const float4*>(res_ptr[i] + ch * col_step));
+      for (int i = 0; i < 4; ++i) {
+        const int r = 8 * i + rsub;
+        float* dst = slot + r * EPI_NC + 4 * (cj ^ ((r >> 1) & 3));
+        if (res_ptr[i]) cp_async16(dst, res_ptr[i] + ch * col_step);
+        else *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);   // a pad token's residual input is zero
+      }
     }
+    cp_async_commit();
   };
-  if (n_chunks > 0) fetch(0, res);
-  if (!acc_ready()) return false;
+  if (MODE != EPI_MERGE) {
+#pragma unroll
+    for (int ch = 0; ch < RES_SLOTS; ++ch) fetch(ch);
+  }
+  if (!acc_ready()) { cp_async_wait<0>(); return false; }
   auto chunk = [&](int ch, const int32_t (&acc)[EPI_NC]) {
     const int n0 = n_first + ch * col_step;
     float v[EPI_NC];
     dequant16<MODE, TAPS>(br, N, m, row_ok, n0, ch * EPI_NC, cc, acc, v);
-    if (ch + 1 < n_chunks) fetch(ch + 1, res_next);
     // row `lane`, logical 16-byte piece j is stored at piece j ^ ((lane >> 1) & 3): conflict-free both ways
 #pragma unroll
     for (int j = 0; j < 4; ++j)
       *reinterpret_cast<float4*>(stage + lane * EPI_NC + 4 * (j ^ ((lane >> 1) & 3))) =
           make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    if (MODE != EPI_MERGE) cp_async_wait<RES_SLOTS - 1>();     // this lane's copies of chunk ch have landed
     __syncwarp();
+    const float* slot = res_ring + (ch % RES_SLOTS) * EPI_STAGE_FLOATS;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int r = 8 * i + rsub;
-      const float4 a = *reinterpret_cast<const float4*>(stage + r * EPI_NC + 4 * (cj ^ ((r >> 1) & 3)));
+      const int off = r * EPI_NC + 4 * (cj ^ ((r >> 1) & 3));
+      const float4 a = *reinterpret_cast<const float4*>(stage + off);
       if (dst_ptr[i]) {
         float4 o = a;
         if (MODE != EPI_MERGE) {
-          const float2 lo = __fadd2_rn(make_float2(res[i].x, res[i].y), make_float2(a.x, a.y));
-          const float2 hi = __fadd2_rn(make_float2(res[i].z, res[i].w), make_float2(a.z, a.w));
+          const float4 rr = *reinterpret_cast<const float4*>(slot + off);
+          const float2 lo = __fadd2_rn(make_float2(rr.x, rr.y), make_float2(a.x, a.y));
+          const float2 hi = __fadd2_rn(make_float2(rr.z, rr.w), make_float2(a.z, a.w));
           o = make_float4(lo.x, lo.y, hi.x, hi.y);
         }
         *reinterpret_cast<float4*>(dst_ptr[i] + ch * col_step) = o;
       }
     }
     __syncwarp();
-#pragma unroll
-    for (int i = 0; i < 4; ++i) res[i] = res_next[i];
+    if (MODE != EPI_MERGE) fetch(ch + RES_SLOTS);              // the slot just read is free again
   };
   int32_t acc[EPI_NC], nxt[EPI_NC];
   if (n_chunks > 0) tmem_ld16_issue(taddr, nxt);
@@ -202,6 +226,7 @@ __device__ __forceinline__ bool epilogue_warp_tile(const GemmBranch& br, int N, 
     if (ch + 1 < n_chunks) tmem_ld16_issue(taddr + (uint32_t)((ch + 1) * col_step), nxt);
     chunk(ch, acc);
   }
+  if (MODE != EPI_MERGE) cp_async_wait<0>();                   // nothing of this tile is left in flight
   return true;
 }
 

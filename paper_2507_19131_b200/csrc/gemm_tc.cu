@@ -41,22 +41,24 @@ struct TcParams {
   int tiles_m0;          // 128-row tiles of the first (high) branch
   int total_tiles, n_tiles, BN, k_blocks, ring, tmem_cols;
   int packed_bytes;      // bytes of the packed staging slot of a stage (0: no branch stages packed rows by TMA)
+  int res_bytes;         // bytes of the residual rings (proj, fc2: RES_SLOTS chunks per epilogue warp; else 0)
   int tma_packed[2];     // branch i stages its bit-packed rows by TMA (tmA_i then describes the packed matrix)
   int* status;
 };
 
 // shared-memory carve-up (offsets from the 1024-byte aligned base)
 struct SmemLayout {
-  int stage_bytes, ring_bytes, consts_off, stage_off, bars_off, total;
+  int stage_bytes, ring_bytes, consts_off, stage_off, res_off, bars_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_bytes) {
+__host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_bytes, int res_bytes) {
   constexpr int NUM_EPI_WARPS = MAX_EPI_WARPS;
   SmemLayout L;
   L.stage_bytes = A_STAGE_BYTES + BN * BK + packed_bytes;
   L.ring_bytes = ring * L.stage_bytes;
   L.consts_off = L.ring_bytes;                                  // per epilogue warp (zc, mult, bias) x 128 columns
   L.stage_off = L.consts_off + NUM_EPI_WARPS * 3 * EPI_WARP_COLS * 4;   // per epilogue warp 32 x 16 floats
-  L.bars_off = L.stage_off + NUM_EPI_WARPS * EPI_STAGE_FLOATS * 4;
+  L.res_off = L.stage_off + NUM_EPI_WARPS * EPI_STAGE_FLOATS * 4;       // residual rings of the binary32 epilogues
+  L.bars_off = L.res_off + res_bytes;
   L.total = L.bars_off + (3 * MAX_RING + 5) * 8 + 16;   // + the drain barrier; then TMEM base, abort flag, fill count
   return L;
 }
@@ -139,7 +141,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
   uint8_t* smem = smem_raw + (base - raw);
-  const SmemLayout L = smem_layout(p.BN, p.ring, p.packed_bytes);
+  const SmemLayout L = smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes);
   const int stage_bytes = L.stage_bytes;
   int32_t* s_consts = reinterpret_cast<int32_t*>(smem + L.consts_off);
   float* s_stage = reinterpret_cast<float*>(smem + L.stage_off);
@@ -305,6 +307,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     // ---- epilogue warps: warp e reads TMEM lanes 32*(e%4).. and takes every EPI_SPLIT-th 16-column chunk ----
     const int e = warp - FIRST_EPI_WARP, q = warp & 3, sub = e >> 2;   // any 4 consecutive warps cover the 4 lane quarters
     float* stage = s_stage + e * EPI_STAGE_FLOATS;
+    float* res_ring = reinterpret_cast<float*>(smem + L.res_off) + e * RES_SLOTS * EPI_STAGE_FLOATS;
     int32_t* c_zc = s_consts + e * 3 * EPI_WARP_COLS;
     float* c_mult = reinterpret_cast<float*>(c_zc + EPI_WARP_COLS);
     float* c_bias = c_mult + EPI_WARP_COLS;
@@ -348,7 +351,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
         return true;
       };
       if (!epilogue_warp_tile<MODE, TAPS>(br, p.g.N, p.g.C, row0, lane, n_tile0, sub, EPI_SPLIT, c_total, cc, taddr, stage,
-                                    acc_ready)) break;
+                                    acc_ready, res_ring)) break;
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * a);
@@ -467,8 +470,9 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
     p.tma_packed[i] = g.br[i].M > 0 && bits != 8 && ((long)g.K * bits / 8) % 16 == 0;
     if (p.tma_packed[i]) p.packed_bytes = BM * (BK / 2);        // room for the widest packed format (4 bit)
   }
+  p.res_bytes = (g.mode == EPI_PROJ || g.mode == EPI_FC2) ? epi_warps(g.mode) * RES_SLOTS * EPI_STAGE_FLOATS * 4 : 0;
   p.ring = MAX_RING;
-  while (p.ring > 2 && smem_layout(p.BN, p.ring, p.packed_bytes).total + 1024 > 220 * 1024) --p.ring;
+  while (p.ring > 2 && smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes).total + 1024 > 220 * 1024) --p.ring;
   p.tmem_cols = 32;
   while (p.tmem_cols < 2 * p.BN) p.tmem_cols <<= 1;
   CUtensorMap mA[2], mB;
@@ -485,7 +489,7 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
     if (!ok) return false;
   }
   if (!make_map(&mB, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN)) return false;
-  const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes).total + 1024 /*alignment slack*/;
+  const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes).total + 1024 /*alignment slack*/;
   // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles)
   int grid = p.total_tiles < sms ? p.total_tiles : sms;
   if (grid > p.n_tiles && grid < p.total_tiles) grid -= grid % p.n_tiles;
