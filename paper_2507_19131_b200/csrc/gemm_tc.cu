@@ -490,9 +490,13 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   }
   if (!make_map(&mB, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN)) return false;
   const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes).total + 1024 /*alignment slack*/;
-  // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles)
+  // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles);
+  // taken only where it does not cost a wave of tiles
   int grid = p.total_tiles < sms ? p.total_tiles : sms;
-  if (grid > p.n_tiles && grid < p.total_tiles) grid -= grid % p.n_tiles;
+  if (grid > p.n_tiles && grid < p.total_tiles) {
+    const int g2 = grid - grid % p.n_tiles;
+    if ((p.total_tiles + g2 - 1) / g2 == (p.total_tiles + grid - 1) / grid) grid = g2;
+  }
   if (g.br[0].tap_acc || g.br[1].tap_acc)
     k_gemm_tc<MODE, true><<<grid, 32 * (2 + unpack_warps(MODE) + epi_warps(MODE)), smem, st>>>(mA[0], mA[1], mB, p);
   else
