@@ -68,6 +68,14 @@ typedef struct {
   float score_inv_scale;                  /* score code = clamp(rne(x * score_inv_scale), -127, 127)       */
   void* prepared;                         /* device buffer of mixaq_block_prepared_bytes(), filled once by */
                                           /* mixaq_block_prepare(); read by every forward call             */
+  int byte_codes;                         /* storage of the block's intermediate activation codes in the workspace.
+                                             0: bit-packed at the branch's bit width (the default; a 4-bit branch
+                                             moves half the bytes of an 8-bit one).  1: one code per byte whatever
+                                             the bit width -- the same code values in [0, 2^bits), no expansion in
+                                             shared memory before the integer MMAs; for maps with many channels,
+                                             where one row tile is read by many column tiles and the codes stay in
+                                             L2, that expansion costs more than the bytes save.  Taps then hold one
+                                             code per byte too.  Workspace sizes depend on this field. */
 } mixaq_block_params;
 
 /* Patch merging between stages: 2x2 neighbours concatenated (zero padding for odd sizes) -> LN(4C) ->
@@ -98,7 +106,7 @@ typedef struct {
 
 /* Optional debug taps of one branch (each pointer may be NULL).  Rows are in window-batch order: window slot
  * s = image * n_branch + rank-within-branch, row = s*49 + in-window token.  Code tensors are bit-packed at the
- * branch's bit width; accumulators are zero-point corrected int32. */
+ * branch's bit width (one code per byte when the block's byte_codes is set); accumulators are zero-point corrected int32. */
 typedef struct {
   uint8_t* a_codes;   int32_t* qkv_acc;  uint8_t* qkv_codes;
   float*   probs;     /* [slots][heads][49][49], the binary32 softmax output before its quantizer */

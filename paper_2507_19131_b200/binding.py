@@ -55,7 +55,7 @@ class BlockS(C.Structure):
     _fields_ = [("dim", C.c_int), ("heads", C.c_int), ("window", C.c_int), ("shift", C.c_int), ("hidden", C.c_int),
                 ("qkv", LinearS), ("proj", LinearS), ("fc1", LinearS), ("fc2", LinearS),
                 ("relpos_table", C.c_void_p), ("hi", BranchS), ("lo", BranchS),
-                ("score_inv_scale", C.c_float), ("prepared", C.c_void_p)]
+                ("score_inv_scale", C.c_float), ("prepared", C.c_void_p), ("byte_codes", C.c_int)]
 
 
 class MergeS(C.Structure):
@@ -256,8 +256,9 @@ def _branch(dev: _Dev, b, cache) -> BranchS:
     return s
 
 
-def fill_block_struct(dev: _Dev, blk) -> BlockS:
+def fill_block_struct(dev: _Dev, blk, byte_codes: bool = False) -> BlockS:
     s = BlockS()
+    s.byte_codes = 1 if byte_codes else 0
     s.dim, s.heads, s.window, s.shift, s.hidden = blk.dim, blk.heads, blk.window, blk.shift, blk.hidden
     s.qkv, s.proj, s.fc1, s.fc2 = (_linear(dev, getattr(blk, n)) for n in ("qkv", "proj", "fc1", "fc2"))
     s.relpos_table = dev.up(blk.relpos, np.float32)
@@ -277,10 +278,10 @@ def fill_merge_struct(dev: _Dev, m) -> MergeS:
 class DeviceBlock:
     """Parameters of one Two-Branch Swin Block resident on the device, prepared (mixaq_block_prepare)."""
 
-    def __init__(self, ctx: Context, blk):
+    def __init__(self, ctx: Context, blk, byte_codes: bool = False):
         self.ctx, self.blk = ctx, blk
         self.dev = _Dev(ctx.device)
-        self.s = fill_block_struct(self.dev, blk)
+        self.s = fill_block_struct(self.dev, blk, byte_codes)
         ctx.check(lib().mixaq_block_prepare(ctx.h, C.byref(self.s), _stream_ptr()), "block_prepare")
         self._ws = None
 
@@ -337,8 +338,8 @@ def block_forward(ctx: Context, db: DeviceBlock, x: torch.Tensor, low_ratio: flo
     tp = None
     if taps:
         n_hi, n_lo, _ = out.counts
-        out.hi, th = _alloc_taps(x.device, B * n_hi * 49, B * n_hi, Cc, db.blk.hidden, db.blk.heads, db.blk.hi.bits)
-        out.lo, tl = _alloc_taps(x.device, B * n_lo * 49, B * n_lo, Cc, db.blk.hidden, db.blk.heads, db.blk.lo.bits)
+        out.hi, th = _alloc_taps(x.device, B * n_hi * 49, B * n_hi, Cc, db.blk.hidden, db.blk.heads, 8 if db.s.byte_codes else db.blk.hi.bits)
+        out.lo, tl = _alloc_taps(x.device, B * n_lo * 49, B * n_lo, Cc, db.blk.hidden, db.blk.heads, 8 if db.s.byte_codes else db.blk.lo.bits)
         tp = Taps(th, tl)
     st = lib().mixaq_block_forward(ctx.h, C.byref(db.s), _ptr(x), _ptr(y), B, H, W, C.c_float(low_ratio),
                                    C.c_float(prune_ratio), C.byref(opts), C.byref(sel) if sel is not None else None,
@@ -470,13 +471,16 @@ def merge_forward_static(ctx: Context, dm: DeviceMerge, x: torch.Tensor, y: torc
 class DeviceBackbone:
     """All parameters of a backbone on the device, prepared; owns the workspace and the stage outputs.
     embed: stem parameters (object with ln_g, ln_b, bias, aq, proj) -- the forward then takes the IMAGE [B,H0,W0,3];
-    norms: one (gamma, beta) pair of numpy vectors per stage -- the stage outputs are then LayerNormed."""
+    norms: one (gamma, beta) pair of numpy vectors per stage -- the stage outputs are then LayerNormed.
+    byte_codes_min_dim: blocks with at least this many channels keep their intermediate codes one per byte
+    (mixaq_block_params.byte_codes); None: every block bit-packs."""
 
-    def __init__(self, ctx: Context, bb, B: int, H0: int, W0: int, embed=None, norms=None):
+    def __init__(self, ctx: Context, bb, B: int, H0: int, W0: int, embed=None, norms=None, byte_codes_min_dim=None):
         self.ctx, self.bb, self.B, self.H0, self.W0 = ctx, bb, B, H0, W0
         self.dev = _Dev(ctx.device)
         nb = len(bb.blocks)
-        self.blocks = (BlockS * nb)(*[fill_block_struct(self.dev, b) for b in bb.blocks])
+        self.blocks = (BlockS * nb)(*[fill_block_struct(self.dev, b, byte_codes_min_dim is not None and b.dim >= byte_codes_min_dim)
+                                      for b in bb.blocks])
         self.merges = (MergeS * max(1, len(bb.merges)))(*[fill_merge_struct(self.dev, m) for m in bb.merges])
         self.depths = (C.c_int * len(bb.depths))(*bb.depths)
         self.s = BackboneS(len(bb.depths), self.depths, self.blocks, self.merges, None, None, None)

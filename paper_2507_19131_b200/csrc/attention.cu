@@ -84,8 +84,8 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
   const bool is_hi = slot < slots_hi;
   const AttnBranch& br = is_hi ? a.br[0] : a.br[1];
   if (!is_hi) slot -= slots_hi;
-  const int bits = br.bits, C = a.C;
-  const long row_bytes = (long)3 * C * bits / 8;
+  const int bits = br.bits, cbits = br.cbits, C = a.C;     // range of a code, bits it occupies in memory
+  const long row_bytes = (long)3 * C * cbits / 8;
   const int zq = br.q.zp, zk = br.k.zp, zv = br.v.zp;
 
   // ---- stage q, k (rows) and v (transposed, permuted) of this head, one code per byte: 3 x 64 row items ----
@@ -93,9 +93,9 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
   if (SHIFTED) { const int w = br.win[slot]; wy = w / a.nwx; wx = w - wy * a.nwx; }
   for (int item = threadIdx.x; item < 3 * 64; item += ATT_WARPS * 32) {
     const int sec = item >> 6, r = item & 63;
-    const uint8_t* src = br.qkv + ((long)slot * WT + r) * row_bytes + (long)(sec * C + h * HEAD_DIM) * bits / 8;
+    const uint8_t* src = br.qkv + ((long)slot * WT + r) * row_bytes + (long)(sec * C + h * HEAD_DIM) * cbits / 8;
     uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    if (r < WT) load_codes_32(src, bits, w);
+    if (r < WT) load_codes_32(src, cbits, w);
     if (sec < 2) {
       int s = 0;
 #pragma unroll
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
   const float kLog2e = 1.44269504088896340736f;
   const float4* relf = reinterpret_cast<const float4*>(a.relbias) + (long)h * (4 * 7 * 32) + lane;
   const long m_base = (long)slot * WT;
-  const long out_row_bytes = (long)C * bits / 8;
+  const long out_row_bytes = (long)C * cbits / 8;
 
   {
     const int mt = warp;
@@ -289,14 +289,14 @@ __global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
       if (i < WT) {
         const uint4 w0 = *reinterpret_cast<const uint4*>(&sm.o[warp][lane][0]);
         const uint4 w1 = *reinterpret_cast<const uint4*>(&sm.o[warp][lane][4]);
-        uint8_t* dst = br.out + (m_base + i) * out_row_bytes + (long)h * HEAD_DIM * bits / 8;
-        if (bits == 8) {
+        uint8_t* dst = br.out + (m_base + i) * out_row_bytes + (long)h * HEAD_DIM * cbits / 8;
+        if (cbits == 8) {
           reinterpret_cast<uint4*>(dst)[0] = w0;
           reinterpret_cast<uint4*>(dst)[1] = w1;
         } else {
           const uint32_t n0 = pack_nibbles(w0.x, w0.y), n1 = pack_nibbles(w0.z, w0.w);
           const uint32_t n2 = pack_nibbles(w1.x, w1.y), n3 = pack_nibbles(w1.z, w1.w);
-          if (bits == 4) {
+          if (cbits == 4) {
             reinterpret_cast<uint4*>(dst)[0] = make_uint4(n0, n1, n2, n3);
           } else {
             reinterpret_cast<uint2*>(dst)[0] = make_uint2(squeeze_pairs(n0) | (squeeze_pairs(n1) << 16),

@@ -29,7 +29,7 @@ constexpr int A_STAGE_BYTES = BM * BK;
 // warps 2..5 expand sub-byte codes (two warps left the long-K main loops of 4-bit tiles waiting for the expansion;
 // eight cost more registers than they return)
 __host__ __device__ constexpr int unpack_warps(int mode) { return 4; }
-constexpr int MAX_EPI_WARPS = 16;              // epilogue warps: 12 for the arithmetic-bound code epilogues, 8 for the binary32 ones
+// epilogue warps: 12 for the arithmetic-bound code epilogues, 8 for the binary32 ones
 __host__ __device__ constexpr int epi_warps(int mode) { return (mode == EPI_QKV || mode == EPI_FC1) ? 12 : 8; }
 constexpr int MAX_BN = 256;
 constexpr int EPI_WARP_COLS = MAX_BN / 2;      // most columns one epilogue warp handles per tile (two warps per lane quarter)
@@ -50,8 +50,7 @@ struct TcParams {
 struct SmemLayout {
   int stage_bytes, ring_bytes, consts_off, stage_off, res_off, bars_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_bytes, int res_bytes) {
-  constexpr int NUM_EPI_WARPS = MAX_EPI_WARPS;
+__host__ __device__ inline SmemLayout smem_layout(int BN, int ring, int packed_bytes, int res_bytes, int NUM_EPI_WARPS) {
   SmemLayout L;
   L.stage_bytes = A_STAGE_BYTES + BN * BK + packed_bytes;
   L.ring_bytes = ring * L.stage_bytes;
@@ -141,7 +140,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
   uint8_t* smem = smem_raw + (base - raw);
-  const SmemLayout L = smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes);
+  const SmemLayout L = smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes, epi_warps(MODE));
   const int stage_bytes = L.stage_bytes;
   int32_t* s_consts = reinterpret_cast<int32_t*>(smem + L.consts_off);
   float* s_stage = reinterpret_cast<float*>(smem + L.stage_off);
@@ -472,7 +471,7 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
   }
   p.res_bytes = (g.mode == EPI_PROJ || g.mode == EPI_FC2) ? epi_warps(g.mode) * RES_SLOTS * EPI_STAGE_FLOATS * 4 : 0;
   p.ring = MAX_RING;
-  while (p.ring > 2 && smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes).total + 1024 > 220 * 1024) --p.ring;
+  while (p.ring > 2 && smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes, epi_warps(MODE)).total + 1024 > 220 * 1024) --p.ring;
   p.tmem_cols = 32;
   while (p.tmem_cols < 2 * p.BN) p.tmem_cols <<= 1;
   CUtensorMap mA[2], mB;
@@ -489,7 +488,8 @@ bool launch_mode(const GemmArgs& g, int* status, cudaStream_t st) {
     if (!ok) return false;
   }
   if (!make_map(&mB, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint32_t)p.BN)) return false;
-  const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes).total + 1024 /*alignment slack*/;
+  const size_t smem = (size_t)smem_layout(p.BN, p.ring, p.packed_bytes, p.res_bytes, epi_warps(MODE)).total + 1024 /*alignment slack*/;
+  if (smem > 227 * 1024) return false;
   // a grid that is a multiple of the number of column tiles keeps every CTA on one column tile (t mod n_tiles);
   // taken only where it does not cost a wave of tiles
   int grid = p.total_tiles < sms ? p.total_tiles : sms;

@@ -87,11 +87,12 @@ bool gemm_init();   // once per device context, before the first launch
 
 // ---- fused window attention ----------------------------------------------------------------------
 struct AttnBranch {
-  const uint8_t* qkv;        // [M][3C*bits/8]
-  uint8_t* out;              // [M][C*bits/8]
+  const uint8_t* qkv;        // [M][3C*cbits/8]
+  uint8_t* out;              // [M][C*cbits/8]
   const int32_t* win;        // [slots] window index (for the shift mask)
   AQ q, k, v, o;
-  int bits, slots;
+  int bits, slots;           // bits: width of the codes' range (and of the probability quantizer)
+  int cbits;                 // bits a stored code occupies: `bits` (bit-packed) or 8 (one code per byte)
   float alpha;               // s_q*s_k/sqrt(d)
   float so;                  // s_p*s_v
   uint8_t* tap_p;            // nullable

@@ -128,6 +128,7 @@ mixaq_status validate_block(mixaq_ctx* ctx, const mixaq_block_params* p, bool ne
       !linear_ok(p->fc1, p->hidden, p->dim) || !linear_ok(p->fc2, p->dim, p->hidden))
     return fail(ctx, MIXAQ_INVALID_ARG, "weight matrix missing or of the wrong shape");
   if (!p->relpos_table) return fail(ctx, MIXAQ_INVALID_ARG, "relpos_table is NULL");
+  if (p->byte_codes != 0 && p->byte_codes != 1) return fail(ctx, MIXAQ_INVALID_ARG, "byte_codes must be 0 or 1");
   if (!need_quantizers) {
     if (!branch_ptrs_ok(p->hi) || !branch_ptrs_ok(p->lo)) return fail(ctx, MIXAQ_INVALID_ARG, "branch parameters invalid");
     return MIXAQ_OK;
@@ -192,7 +193,7 @@ BlockWs carve_block(const mixaq_block_params* p, int B, int H, int W, void* base
   w.sel = carve_sel(B, H, W, base ? (char*)base + c.off : nullptr);
   c.off += w.sel.bytes;
   for (int i = 0; i < 2; ++i) {
-    const int bits = i == 0 ? p->hi.bits : p->lo.bits;
+    const int bits = p->byte_codes ? 8 : (i == 0 ? p->hi.bits : p->lo.bits);     // container of a code
     w.a[i]   = c.take<uint8_t>(rows * C * bits / 8);
     w.qkv[i] = c.take<uint8_t>(rows * 3 * C * bits / 8);
     w.o[i]   = c.take<uint8_t>(rows * C * bits / 8);
@@ -458,12 +459,14 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   const int M[2] = {B * g.n_hi * WT, B * g.n_lo * WT};
   const int slots[2] = {B * g.n_hi, B * g.n_lo};
   const mixaq_branch_taps* tp[2] = {taps ? &taps->hi : nullptr, taps ? &taps->lo : nullptr};
+  // bits a stored code occupies: the branch's bit width (bit-packed) or a whole byte
+  const int cb[2] = {p->byte_codes ? 8 : p->hi.bits, p->byte_codes ? 8 : p->lo.bits};
 
   // 2. gather + LN1 + quantize + pack
   LnBranch lb[2];
   for (int i = 0; i < 2; ++i) {
     lb[i].src = x; lb[i].rowsrc = sel.rowsrc[i]; lb[i].gamma = brp[i]->ln1_g; lb[i].beta = brp[i]->ln1_b;
-    lb[i].out = ws.a[i]; lb[i].q = to_aq(brp[i]->qkv_in); lb[i].M = M[i];
+    lb[i].out = ws.a[i]; lb[i].q = to_aq(brp[i]->qkv_in); lb[i].q.bits = cb[i]; lb[i].M = M[i];
   }
   { PROF(PC_LN1); launch_ln_quant(lb[0], lb[1], C, st); }
 
@@ -472,9 +475,9 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   ga.status = ctx->d_status;
   ga.w = p->qkv.codes; ga.N = 3 * C; ga.K = C; ga.C = C; ga.mode = EPI_QKV;
   for (int i = 0; i < 2; ++i) {
-    fill_gemm_branch(ga.br[i], ws.a[i], M[i], brp[i]->bits, pr.mult[0][i], pr.zc[0][i], brp[i]->b_qkv);
+    fill_gemm_branch(ga.br[i], ws.a[i], M[i], cb[i], pr.mult[0][i], pr.zc[0][i], brp[i]->b_qkv);
     ga.br[i].q0 = to_aq(brp[i]->q); ga.br[i].q1 = to_aq(brp[i]->k); ga.br[i].q2 = to_aq(brp[i]->v);
-    ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.qkv[i];
+    ga.br[i].out_bits = cb[i]; ga.br[i].out_codes = ws.qkv[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->qkv_acc : nullptr;
   }
   { PROF(PC_QKV); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
@@ -488,7 +491,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     AttnBranch& ab = aa.br[i];
     ab.qkv = ws.qkv[i]; ab.out = ws.o[i]; ab.win = sel.win[i];
     ab.q = to_aq(brp[i]->q); ab.k = to_aq(brp[i]->k); ab.v = to_aq(brp[i]->v); ab.o = to_aq(brp[i]->proj_in);
-    ab.bits = brp[i]->bits; ab.slots = slots[i];
+    ab.bits = brp[i]->bits; ab.cbits = cb[i]; ab.slots = slots[i];
     ab.alpha = (brp[i]->q.scale * brp[i]->k.scale) * rs;
     ab.so = (1.0f / (float)((1 << brp[i]->bits) - 1)) * brp[i]->v.scale;
     ab.tap_p = tp[i] ? tp[i]->p_codes : nullptr; ab.tap_probs = tp[i] ? tp[i]->probs : nullptr; ab.tap_pv = tp[i] ? tp[i]->pv_acc : nullptr;
@@ -498,7 +501,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   // 5. proj GEMM + attention residual -> x1
   ga.w = p->proj.codes; ga.N = C; ga.K = C; ga.mode = EPI_PROJ;
   for (int i = 0; i < 2; ++i) {
-    fill_gemm_branch(ga.br[i], ws.o[i], M[i], brp[i]->bits, pr.mult[1][i], pr.zc[1][i], brp[i]->b_proj);
+    fill_gemm_branch(ga.br[i], ws.o[i], M[i], cb[i], pr.mult[1][i], pr.zc[1][i], brp[i]->b_proj);
     ga.br[i].out_f = ws.x1[i]; ga.br[i].res = x; ga.br[i].rowsrc = sel.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->proj_acc : nullptr;
   }
@@ -507,15 +510,15 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   // 6. LN2 + quantize + pack
   for (int i = 0; i < 2; ++i) {
     lb[i].src = ws.x1[i]; lb[i].rowsrc = nullptr; lb[i].gamma = brp[i]->ln2_g; lb[i].beta = brp[i]->ln2_b;
-    lb[i].out = ws.f1[i]; lb[i].q = to_aq(brp[i]->fc1_in); lb[i].M = M[i];
+    lb[i].out = ws.f1[i]; lb[i].q = to_aq(brp[i]->fc1_in); lb[i].q.bits = cb[i]; lb[i].M = M[i];
   }
   { PROF(PC_LN2); launch_ln_quant(lb[0], lb[1], C, st); }
 
   // 7. fc1 GEMM + GELU + requantize
   ga.w = p->fc1.codes; ga.N = Hd; ga.K = C; ga.mode = EPI_FC1;
   for (int i = 0; i < 2; ++i) {
-    fill_gemm_branch(ga.br[i], ws.f1[i], M[i], brp[i]->bits, pr.mult[2][i], pr.zc[2][i], brp[i]->b_fc1);
-    ga.br[i].q0 = to_aq(brp[i]->fc2_in); ga.br[i].out_bits = brp[i]->bits; ga.br[i].out_codes = ws.f2[i];
+    fill_gemm_branch(ga.br[i], ws.f1[i], M[i], cb[i], pr.mult[2][i], pr.zc[2][i], brp[i]->b_fc1);
+    ga.br[i].q0 = to_aq(brp[i]->fc2_in); ga.br[i].out_bits = cb[i]; ga.br[i].out_codes = ws.f2[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc1_acc : nullptr;
   }
   { PROF(PC_FC1); if (!launch_gemm(ga, st)) return fail(ctx, MIXAQ_INTERNAL, "GEMM launch set-up failed (tensor map / tile shape)"); }
@@ -523,7 +526,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   // 8. fc2 GEMM + residual + scatter (reverse shift, crop)
   ga.w = p->fc2.codes; ga.N = C; ga.K = Hd; ga.mode = EPI_FC2;
   for (int i = 0; i < 2; ++i) {
-    fill_gemm_branch(ga.br[i], ws.f2[i], M[i], brp[i]->bits, pr.mult[3][i], pr.zc[3][i], brp[i]->b_fc2);
+    fill_gemm_branch(ga.br[i], ws.f2[i], M[i], cb[i], pr.mult[3][i], pr.zc[3][i], brp[i]->b_fc2);
     ga.br[i].out_f = y; ga.br[i].res = ws.x1[i]; ga.br[i].rowsrc = sel.rowsrc[i];
     ga.br[i].tap_acc = tp[i] ? tp[i]->fc2_acc : nullptr;
   }
@@ -534,7 +537,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
 
   if (taps) {
     for (int i = 0; i < 2; ++i) {
-      const size_t rows = (size_t)M[i]; const int bits = brp[i]->bits;
+      const size_t rows = (size_t)M[i]; const int bits = cb[i];
       if (rows == 0) continue;
       if (tp[i]->a_codes)   cudaMemcpyAsync(tp[i]->a_codes, ws.a[i], rows * C * bits / 8, cudaMemcpyDeviceToDevice, st);
       if (tp[i]->qkv_codes) cudaMemcpyAsync(tp[i]->qkv_codes, ws.qkv[i], rows * 3 * C * bits / 8, cudaMemcpyDeviceToDevice, st);
@@ -714,7 +717,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
       put_lin(q.qkv); put_lin(q.proj); put_lin(q.fc1); put_lin(q.fc2);
       put(&q.relpos_table, sizeof(q.relpos_table));
       put_branch(q.hi); put_branch(q.lo);
-      put(&q.score_inv_scale, 4); put(&q.prepared, sizeof(q.prepared));
+      put(&q.score_inv_scale, 4); put(&q.prepared, sizeof(q.prepared)); put(&q.byte_codes, 4);
     }
     for (int m = 0; m + 1 < p->num_stages; ++m) {
       const mixaq_merge_params& q = p->merges[m];

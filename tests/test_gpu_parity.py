@@ -39,13 +39,13 @@ def assert_close_rel(got, want, tol=TOL):
     assert err <= tol * scale, f"max abs err {err} > {tol} * {scale}"
 
 
-def check_taps(orc, blk, ref, got, counts):
-    """Every intermediate of both branches, bit for bit."""
+def check_taps(orc, blk, ref, got, counts, byte_codes=False):
+    """Every intermediate of both branches, bit for bit (byte_codes: the block stores one code per byte)."""
     for name, br, n in (("hi", blk.hi, counts[0]), ("lo", blk.lo, counts[1])):
         r, g = getattr(ref, name), getattr(got, name)
         if n == 0:
             continue
-        bits = br.bits
+        bits = 8 if byte_codes else br.bits
         for f in ("a_codes", "qkv_codes", "o_codes", "f1_codes", "f2_codes"):
             assert np.array_equal(g.__dict__[f].cpu().numpy(), orc.pack(r.__dict__[f], bits)), f"{name}.{f}"
         for f in ("qkv_acc", "pv_acc", "proj_acc", "fc1_acc", "fc2_acc", "p_codes"):
@@ -56,10 +56,10 @@ def check_taps(orc, blk, ref, got, counts):
         assert np.array_equal(g.x1.cpu().numpy(), r.x1), f"{name}.x1 not bit-identical"
 
 
-def run_block_case(orc, mq, ctx, blk, x, low, prune=0.0, reverse=False, stage_energy=False, taps=True):
+def run_block_case(orc, mq, ctx, blk, x, low, prune=0.0, reverse=False, stage_energy=False, taps=True, byte_codes=False):
     # the C ABI takes the ratios as binary32: both sides get exactly that value (0.11f * 6000 is below 660)
     low, prune = float(F32(low)), float(F32(prune))
-    db = mq.DeviceBlock(ctx, blk)
+    db = mq.DeviceBlock(ctx, blk, byte_codes=byte_codes)
     xd = dev(x)
     e_ref = e_dev = None
     if stage_energy:
@@ -79,7 +79,7 @@ def run_block_case(orc, mq, ctx, blk, x, low, prune=0.0, reverse=False, stage_en
         for b in range(x.shape[0]):
             assert np.array_equal(lst[b], np.flatnonzero(ref.cls[b] == c)), f"class {c} list of image {b}"
     if taps:
-        check_taps(orc, blk, ref, got, ref.counts)
+        check_taps(orc, blk, ref, got, ref.counts, byte_codes)
     y = got.y.cpu().numpy()
     assert_close_rel(y, ref.y)
     assert np.array_equal(y, ref.y), "outputs are within tolerance but not bit-identical"
@@ -111,6 +111,15 @@ def test_block_tiny_all_taps(orc, mq, ctx, shift, bits):
     blk = synth.make_block(np.random.default_rng(10 + shift), 64, 2, shift, 4, bits[0], bits[1], share_bias=False)
     x = synth.input_blobs(11, 2, 17, 23, 64, bg_std=0.5, gain=4.0)     # ragged: padded to 21 x 28
     run_block_case(orc, mq, ctx, blk, x, 0.4, stage_energy=bool(shift))
+
+
+@pytest.mark.parametrize("dim,bits", [(64, (8, 4)), (64, (4, 2)), (384, (8, 4)), (192, (8, 2))])
+def test_block_one_code_per_byte_all_taps(orc, mq, ctx, dim, bits):
+    """byte_codes = 1: the same code values, stored one per byte whatever the bit width; every tap and the output as
+    before (the oracle's codes, here compared unpacked)."""
+    blk = synth.make_block(np.random.default_rng(dim + bits[1]), dim, dim // 32, 3, 4, bits[0], bits[1], share_bias=False)
+    x = synth.input_blobs(12, 2, 17, 23, dim, bg_std=0.5, gain=4.0)
+    run_block_case(orc, mq, ctx, blk, x, 0.4, 0.1, byte_codes=True)
 
 
 def test_block_config1_all_taps(orc, mq, ctx):
@@ -266,16 +275,19 @@ def _full_backbone_case(orc, mq, ctx, wl):
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
-        dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
         xd = dev(wl.x)
-        for call in range(2):
-            got = mq.backbone_forward(ctx, dbb, xd, wl.low_ratios, wl.prune_ratios)
-            side.synchronize()
-            assert ctx.device_status() == 0
-            for st, (g, w) in enumerate(zip(got, want)):
-                g = g.cpu().numpy()
-                assert_close_rel(g, w)
-                assert np.array_equal(g, w), f"stage {st} (call {call}) within tolerance but not bit-identical"
+        # every block bit-packed, then the storage the benchmark uses (one code per byte from 384 channels on)
+        for byte_min in (None, 384):
+            dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W, byte_codes_min_dim=byte_min)
+            for call in range(2):
+                got = mq.backbone_forward(ctx, dbb, xd, wl.low_ratios, wl.prune_ratios)
+                side.synchronize()
+                assert ctx.device_status() == 0
+                for st, (g, w) in enumerate(zip(got, want)):
+                    g = g.cpu().numpy()
+                    assert_close_rel(g, w)
+                    assert np.array_equal(g, w), f"stage {st} (call {call}, byte codes from {byte_min}) not bit-identical"
+            del dbb
     torch.cuda.current_stream().wait_stream(side)
 
 
