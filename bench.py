@@ -192,6 +192,8 @@ def run_ours(args):
     torch.cuda.set_stream(torch.cuda.Stream())
     ctx = mq.Context(local)
     K, Wm = args.steps, max(args.warmup, 3)
+    # storage of the blocks' intermediate codes: bit-packed below this many channels, one code per byte from there on
+    BYTE_MIN = args.byte_codes_min_dim if args.byte_codes_min_dim > 0 else None
 
     def barrier():
         if world > 1:
@@ -200,11 +202,12 @@ def run_ours(args):
 
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
-    def time_ratio(ratio, steps, warm, sampler=None, e2e=False):
+    def time_ratio(ratio, steps, warm, sampler=None, e2e=False, byte_min="default"):
+        byte_min = BYTE_MIN if byte_min == "default" else byte_min
         wl = workload(ratio)
         # replicas differ only in their seed-shifted input (weak scaling: one image per rank per step)
         x_host = torch.from_numpy(replicas.rank_input(wl.x, rank)).pin_memory()
-        dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+        dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W, byte_codes_min_dim=byte_min)
         x_dev = x_host.cuda()
         outs_host = [torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in dbb.outs]
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
@@ -244,7 +247,7 @@ def run_ours(args):
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
         sets = []
         for _ in range(2):
-            dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W)
+            dbb = mq.DeviceBackbone(ctx, wl.backbone, wl.B, wl.H, wl.W, byte_codes_min_dim=BYTE_MIN)
             sets.append(dict(dbb=dbb, x=torch.empty_like(x_host, device="cuda"),
                              host=[torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in dbb.outs],
                              e_in=torch.cuda.Event(), e_comp=torch.cuda.Event(), e_out=torch.cuda.Event()))
@@ -376,6 +379,13 @@ def run_ours(args):
     e2e = time_e2e(args.ratio, K, Wm)
     e2e_value = replicas.job_throughput(wl_images(e2e["wl"]), K, world, e2e["ms"])
 
+    # the same forward with every block's codes bit-packed (what the expansion in shared memory costs in stages 3-4)
+    packed_value = None
+    if BYTE_MIN is not None and world == 1:
+        n_p = max(3, K // 2)
+        s_p = time_ratio(args.ratio, n_p, 3, byte_min=None)
+        packed_value = round(wl_images(s_p["wl"]) * n_p / (s_p["ms"] / 1e3), 2)
+
     sweep = {}
     if args.sweep and world == 1:
         for r in SWEEP_BY_CONFIG[CONFIG]:
@@ -402,7 +412,7 @@ def run_ours(args):
         wl_s = main["wl"]
         emb = synth.make_embed(rng, bbm.dims[0])
         norms = [(np.ones(c, np.float32), np.zeros(c, np.float32)) for c in bbm.dims]
-        dbs = mq.DeviceBackbone(ctx, wl_s.backbone, wl_s.B, 800, 1333, embed=emb, norms=norms)
+        dbs = mq.DeviceBackbone(ctx, wl_s.backbone, wl_s.B, 800, 1333, embed=emb, norms=norms, byte_codes_min_dim=BYTE_MIN)
         img = torch.from_numpy(synth.input_image(78, wl_s.B, 800, 1333)).cuda()
         for _ in range(3):
             mq.backbone_forward(ctx, dbs, img, wl_s.low_ratios, wl_s.prune_ratios)
@@ -445,6 +455,8 @@ def run_ours(args):
                    "weights": "W%d (int8 container)" % bbm.blocks[0].qkv.bits,
                    "act_bits_high_low": [bbm.blocks[0].hi.bits, bbm.blocks[0].lo.bits], "low_ratio": args.ratio,
                    "prune_ratio": (main["wl"].prune_ratios or [0.0])[0],
+                   "code_storage": ("bit-packed in every block" if BYTE_MIN is None else
+                                    f"bit-packed in blocks of fewer than {BYTE_MIN} channels, one code per byte from {BYTE_MIN} on"),
                    "l2": f"flushed between timed iterations ({L2_FLUSH_BYTES >> 20} MiB write)",
                    "parallelism": "replicas only (one image per GPU, no collective)"},
         "clocks": main["clocks"],
@@ -458,6 +470,7 @@ def run_ours(args):
         "gpu_launches": main["launches"] * K,
         "roofline": roof,
         "kernels": kernels,
+        "value_all_bit_packed": packed_value,
         "low_ratio_sweep_images_per_sec": sweep,
         "paper_cost_model": cost,
         "value_with_stem": stem,
@@ -590,6 +603,9 @@ def main():
     ap.add_argument("--sweep", dest="force_sweep", action="store_true",
                     help="also sweep the low-bit ratio for --config 4 (0 ... 0.75) or 5 (0 ... 0.8); config 3 sweeps by default")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--byte-codes-min-dim", type=int, default=384,
+                    help="blocks with at least this many channels store their intermediate codes one per byte "
+                         "(mixaq_block_params.byte_codes); 0: every block bit-packs")
     args = ap.parse_args()
     global CONFIG
     CONFIG = args.config

@@ -73,7 +73,7 @@ __device__ __forceinline__ uint32_t squeeze_pairs(uint32_t t) {
 
 // TAPS: the debug taps (softmax output, P codes, P.V accumulators) are compiled in only for calls that ask for them
 template <bool SHIFTED, bool TAPS>
-__global__ void __launch_bounds__(ATT_WARPS * 32, 7) k_attention(AttnArgs a) {
+__global__ void __launch_bounds__(ATT_WARPS * 32, 8) k_attention(AttnArgs a) {
   __shared__ __align__(16) WarpSmem sm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
