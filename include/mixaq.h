@@ -268,6 +268,12 @@ mixaq_status mixaq_set_window_elevation(mixaq_ctx* ctx, int allow);
  * mixaq_select_opts. */
 mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse);
 
+/* NVTX ranges for external tracers (off by default): every kernel family launched through this context is wrapped in
+ * a host-side range named like its profiling category, and mixaq_backbone_forward adds one range per stage and per
+ * block.  The ranges mark where the launches are ISSUED: a forward that replays a cached graph issues none, so trace
+ * with the graph cache off (mixaq_set_graph_cache) to see them. */
+mixaq_status mixaq_set_nvtx(mixaq_ctx* ctx, int enabled);
+
 /* Number of kernel launches the last block / merge / backbone call of this context issued. */
 int          mixaq_last_launch_count(const mixaq_ctx* ctx);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
     "mixaq_norm_forward", "mixaq_profile_end_records", "mixaq_calibrate_block_workspace_bytes", "mixaq_calibrate_block",
-    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection",
+    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection", "mixaq_set_nvtx",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
@@ -161,6 +161,10 @@ class Context:
 
     def device_status(self) -> int:
         return lib().mixaq_last_device_status(self.h, _stream_ptr())
+
+    def set_nvtx(self, enabled: bool):
+        """mixaq_set_nvtx: host-side NVTX ranges per kernel family, stage and block."""
+        self.check(lib().mixaq_set_nvtx(self.h, 1 if enabled else 0), "set_nvtx")
 
     def set_reverse_selection(self, reverse: bool):
         self.check(lib().mixaq_set_reverse_selection(self.h, 1 if reverse else 0), "set_reverse_selection")

@@ -33,7 +33,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + sources() + ["-lcuda"]
+    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + sources() + ["-lcuda", "-ldl"]
     # libcuda is only needed for the tensor-map encoder; resolve it lazily so the build works without a driver
     cmd = [c for c in cmd if c != "-lcuda"]
     subprocess.check_call(cmd)

@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/mixaq.h: argument validation, workspace carving, the launch
 // schedule of one Two-Branch Swin Block (MixA-Q Section 3.2, Figure 3) and of the backbone loop.
 // Nothing here computes: every step of the path runs in the kernels.
+#include <nvtx3/nvToolsExt.h>
 #include "../../include/mixaq.h"
 #include "kernels.h"
 #include <cmath>
@@ -29,6 +30,7 @@ struct mixaq_ctx {
   bool profiling;
   bool graph_cache;                    // replay backbone forwards as CUDA graphs (see mixaq_set_graph_cache)
   bool reverse_selection;              // backbone: worst-case selection order (Table 4) in every block
+  bool nvtx;                           // name every kernel family, stage and block with an NVTX range (host side)
   bool allow_elevation;                // backbone: every pair uses its own ratios even if an earlier pair of the stage had larger ones
   std::vector<GraphEntry> graphs;
   std::vector<ProfRec> prof;          // event pairs recorded since mixaq_profile_begin
@@ -82,8 +84,9 @@ mixaq_status check_cuda(mixaq_ctx* ctx, const char* where) {
 
 // Per-kernel CUDA-event timing (only while profiling is on; the events sit on the launching stream).
 struct ProfScope {
-  mixaq_ctx* ctx; cudaStream_t st; cudaEvent_t e1; bool on;
-  ProfScope(mixaq_ctx* c, int cat, cudaStream_t s) : ctx(c), st(s), e1(nullptr), on(c && c->profiling) {
+  mixaq_ctx* ctx; cudaStream_t st; cudaEvent_t e1; bool on, range;
+  ProfScope(mixaq_ctx* c, int cat, cudaStream_t s) : ctx(c), st(s), e1(nullptr), on(c && c->profiling), range(c && c->nvtx) {
+    if (range) nvtxRangePushA(kProfNames[cat]);
     if (!on) return;
     cudaEvent_t ev[2];
     for (int i = 0; i < 2; ++i) {
@@ -94,7 +97,18 @@ struct ProfScope {
     e1 = ev[1];
     ctx->prof.push_back({cat, ev[0], ev[1]});
   }
-  ~ProfScope() { if (on) cudaEventRecord(e1, st); }
+  ~ProfScope() { if (on) cudaEventRecord(e1, st); if (range) nvtxRangePop(); }
+};
+// NVTX range over a stage or a block of the backbone walk (only with mixaq_set_nvtx)
+struct NvtxScope {
+  bool on;
+  NvtxScope(const mixaq_ctx* c, const char* what, int index) : on(c && c->nvtx) {
+    if (!on) return;
+    char name[48];
+    snprintf(name, sizeof(name), "%s %d", what, index);
+    nvtxRangePushA(name);
+  }
+  ~NvtxScope() { if (on) nvtxRangePop(); }
 };
 #define PROF(cat) ProfScope prof_scope_##cat(ctx, cat, st)
 
@@ -245,7 +259,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false; c->nvtx = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
       !gemm_init()) {
     cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
@@ -758,6 +772,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     cur = ws.tokens;
   }
   for (int s = 0; s < p->num_stages && result == MIXAQ_OK; ++s) {
+    NvtxScope stage_range(ctx, "stage", s + 1);
     const int d = p->depths[s];
     // with output norms the un-normalised map stays in the workspace (the next stage reads it) and the caller's
     // buffer receives its LayerNorm
@@ -800,6 +815,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     total += g_launches;
     for (int i = 0; i < d; ++i, ++blk) {
       float* dst = ((d - 1 - i) % 2 == 0) ? out_s : ws.scratch;
+      NvtxScope block_range(ctx, "block", blk);
       result = block_forward_impl(ctx, &p->blocks[blk], cur, dst, B, H, W, lr_eff[i], pr_eff[i], nullptr, nullptr,
                                   ws.block, ws.block_bytes, nullptr, &sels[i], st);
       if (result != MIXAQ_OK) break;
@@ -919,6 +935,12 @@ mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float*
 mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   ctx->reverse_selection = reverse != 0;
+  return MIXAQ_OK;
+}
+
+mixaq_status mixaq_set_nvtx(mixaq_ctx* ctx, int enabled) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  ctx->nvtx = enabled != 0;
   return MIXAQ_OK;
 }
 

@@ -251,6 +251,11 @@ def test_precision_classes_within_a_stage_and_the_elevation_switch(orc, mq):
         got = mq.backbone_forward(c, dbb, dev(x), ratios, prunes)[0].cpu().numpy()
         want = orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=True, reverse=True)[0]
         assert np.array_equal(got, want) and not np.array_equal(got, orc.backbone_forward(bb, x, ratios, prunes, allow_elevation=True)[0])
+        # NVTX ranges around every launch, stage and block (no tracer attached: the calls must be harmless)
+        c.set_nvtx(True)
+        again = mq.backbone_forward(c, dbb, dev(x), ratios, prunes)[0].cpu().numpy()
+        c.set_nvtx(False)
+        assert np.array_equal(again, got)
         assert c.device_status() == 0
     finally:
         c.close()
