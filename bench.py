@@ -314,6 +314,9 @@ def run_ours(args):
     prof = ctx.profile_end()
     work = algorithmic_work(main["wl"], mq)
     kernels = {}
+    # what an event pair adds by itself (pairs with nothing between them, recorded in the same graphs)
+    b_ms, b_cnt = prof.pop("empty_event_bracket", (0.0, 0))
+    bracket_ms = b_ms / b_cnt if b_cnt else 0.0
     for cat, (ms, cnt) in prof.items():
         if cnt == 0:
             continue
@@ -321,7 +324,8 @@ def run_ours(args):
         per_fwd_ms = ms / K
         kernels[cat] = dict(ms_per_step=round(per_fwd_ms, 5), launches_per_step=cnt // K,
                             share=0.0, tops=round(w["ops"] / (per_fwd_ms * 1e-3) / 1e12, 3) if w["ops"] else None,
-                            gbs=round(w["bytes"] / (per_fwd_ms * 1e-3) / 1e9, 1))
+                            gbs=round(w["bytes"] / (per_fwd_ms * 1e-3) / 1e9, 1),
+                            ms_net_of_bracket=round(max(per_fwd_ms - bracket_ms * (cnt // K), 0.0), 5))
     tot = sum(v["ms_per_step"] for v in kernels.values()) or 1.0
     for v in kernels.values():
         v["share"] = round(v["ms_per_step"] / tot, 4)
@@ -350,6 +354,12 @@ def run_ours(args):
                 peak_source=f"2 x bf16_tflops (burst) of {peaks['source']} peaks; sustained: 2 x bf16_tflops_sustained",
                 launches_per_step=gemm_launches, launch_us=round(1e3 * gemm_ms / max(1, gemm_launches), 3),
                 gemm_ms_per_step=round(gemm_ms, 5), gemm_gop_per_step=round(gemm_ops / 1e9, 2),
+                event_bracket_us=round(bracket_ms * 1e3, 3),
+                frac_net_of_bracket=round(gemm_ops / max((gemm_ms - bracket_ms * gemm_launches) * 1e-3, 1e-9) / 1e12 / peak_burst, 5),
+                net_note=("every launch is timed between two event records, which by themselves take event_bracket_us "
+                          "(pairs with nothing between them, same graphs); frac uses the bracketed times as they are, "
+                          "frac_net_of_bracket subtracts that per launch.  Check: the net kernel times of one forward sum to "
+                          f"{sum(v['ms_net_of_bracket'] for v in kernels.values()):.4f} ms against {ms_per_step:.4f} ms per timed forward"),
                 traffic=traffic,
                 traffic_note=("mean dram bytes per GEMM launch (ncu, profiles/ncu_dram_traffic.json)" if traffic is not None else
                               "no ncu record for these kernel sources and this workload"),

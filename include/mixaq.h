@@ -253,7 +253,8 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
  * launches on `cuda_stream`, later calls cost one graph launch on the host.  The data behind the pointers may
  * change freely between calls.  Captured graphs are kept per context (16 at most) until mixaq_destroy.  Caching
  * needs a stream that can be captured: calls on the legacy default stream (NULL), calls made while the caller is
- * capturing the stream itself, and calls between mixaq_profile_begin/end launch their kernels directly.
+ * capturing the stream itself launch their kernels directly.  A call between mixaq_profile_begin/end is captured
+ * together with its event records, launched once and not cached.
  * enabled = 0 switches the cache off and drops the stored graphs; it is on by default. */
 mixaq_status mixaq_set_graph_cache(mixaq_ctx* ctx, int enabled);
 
@@ -294,7 +295,10 @@ mixaq_status mixaq_measure_mma_peak(mixaq_ctx* ctx, int kind, int groups, void* 
  *      Between begin and end every kernel family launched through this context is bracketed by CUDA events on
  *      the launching stream.  end() synchronises the stream and returns, per category (see
  *      mixaq_profile_category_name), the summed device milliseconds and the number of event pairs; both HOST
- *      arrays have mixaq_profile_categories() entries.  Profiling creates events (not graph-capturable). ---- */
+ *      arrays have mixaq_profile_categories() entries.  A backbone forward on a capturable stream is timed as it runs
+ *      inside its graph (the event records are graph nodes); other calls are timed as stream launches, which adds the
+ *      launch gap to every kernel.  Category "empty_event_bracket": four event pairs per backbone
+ *      forward with nothing between them -- what a bracket by itself adds to a kernel's figure. ---- */
 int          mixaq_profile_categories(void);
 const char*  mixaq_profile_category_name(int category);
 mixaq_status mixaq_profile_begin(mixaq_ctx* ctx);

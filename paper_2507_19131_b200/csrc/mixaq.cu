@@ -30,6 +30,8 @@ struct mixaq_ctx {
   bool profiling;
   bool graph_cache;                    // replay backbone forwards as CUDA graphs (see mixaq_set_graph_cache)
   bool reverse_selection;              // backbone: worst-case selection order (Table 4) in every block
+  bool prof_capture;                   // the profiled call is being captured: event records become graph nodes
+  std::vector<cudaGraphExec_t> prof_execs;   // graphs of profiled forwards, destroyed when the profiling ends
   bool nvtx;                           // name every kernel family, stage and block with an NVTX range (host side)
   bool allow_elevation;                // backbone: every pair uses its own ratios even if an earlier pair of the stage had larger ones
   std::vector<GraphEntry> graphs;
@@ -48,11 +50,11 @@ void ctx_note(mixaq_ctx* ctx, const char* msg, int launches) {
 }  // namespace mixaq
 
 enum ProfCat { PC_ENERGY = 0, PC_SELECT, PC_LN1, PC_QKV, PC_ATTN, PC_PROJ, PC_LN2, PC_FC1, PC_FC2, PC_COPY,
-               PC_MERGE_GATHER, PC_MERGE_GEMM, PC_STEM, PC_OUT_NORM, PC_COUNT };
+               PC_MERGE_GATHER, PC_MERGE_GEMM, PC_STEM, PC_OUT_NORM, PC_BRACKET, PC_COUNT };
 static const char* kProfNames[PC_COUNT] = {"energy", "select", "gather_ln1_quant", "gemm_qkv", "attention",
                                            "gemm_proj", "ln2_quant", "gemm_fc1_gelu", "gemm_fc2_scatter",
                                            "copy_pruned", "merge_gather_ln_quant", "gemm_merge", "patch_embed",
-                                           "stage_output_norm"};
+                                           "stage_output_norm", "empty_event_bracket"};
 
 namespace {
 
@@ -93,11 +95,16 @@ struct ProfScope {
       if (!ctx->pool.empty()) { ev[i] = ctx->pool.back(); ctx->pool.pop_back(); }
       else if (cudaEventCreate(&ev[i]) != cudaSuccess) { on = false; return; }
     }
-    cudaEventRecord(ev[0], st);
+    record(ev[0]);
     e1 = ev[1];
     ctx->prof.push_back({cat, ev[0], ev[1]});
   }
-  ~ProfScope() { if (on) cudaEventRecord(e1, st); if (range) nvtxRangePop(); }
+  // inside a stream capture the record becomes a graph node of its own (an "external" event keeps its timestamp)
+  void record(cudaEvent_t e) {
+    if (ctx->prof_capture) cudaEventRecordWithFlags(e, st, cudaEventRecordExternal);
+    else cudaEventRecord(e, st);
+  }
+  ~ProfScope() { if (on) record(e1); if (range) nvtxRangePop(); }
 };
 // NVTX range over a stage or a block of the backbone walk (only with mixaq_set_nvtx)
 struct NvtxScope {
@@ -259,7 +266,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false; c->nvtx = false;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false; c->nvtx = false; c->prof_capture = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
       !gemm_init()) {
     cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
@@ -272,6 +279,7 @@ mixaq_status mixaq_destroy(mixaq_ctx* ctx) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   if (ctx->d_status) cudaFree(ctx->d_status);
   for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
+  for (cudaGraphExec_t g : ctx->prof_execs) cudaGraphExecDestroy(g);
   for (auto& r : ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
   for (auto e : ctx->pool) cudaEventDestroy(e);
   delete ctx;
@@ -339,6 +347,8 @@ mixaq_status mixaq_profile_end(mixaq_ctx* ctx, void* cuda_stream, float* ms_per_
   if (!ctx || !ms_per_category || !launches_per_category) return MIXAQ_INVALID_ARG;
   ctx->profiling = false;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return check_cuda(ctx, "profile_end");
+  for (cudaGraphExec_t g : ctx->prof_execs) cudaGraphExecDestroy(g);
+  ctx->prof_execs.clear();
   for (int i = 0; i < PC_COUNT; ++i) { ms_per_category[i] = 0.f; launches_per_category[i] = 0; }
   for (auto& r : ctx->prof) {
     float ms = 0.f;
@@ -353,6 +363,8 @@ mixaq_status mixaq_profile_end_records(mixaq_ctx* ctx, void* cuda_stream, int* c
   if (!ctx || !category || !ms || !count || capacity < 0) return MIXAQ_INVALID_ARG;
   ctx->profiling = false;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return check_cuda(ctx, "profile_end_records");
+  for (cudaGraphExec_t g : ctx->prof_execs) cudaGraphExecDestroy(g);
+  ctx->prof_execs.clear();
   int n = 0;
   for (auto& r : ctx->prof) {
     float t = 0.f;
@@ -703,13 +715,19 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
 
   // Replay as a CUDA graph when an identical call was captured before.  The key is made of every value that
   // shapes the launches: the fields of the HOST parameter structs, ratios, pointers, sizes and the stream.
-  bool use_graph = ctx->graph_cache && !ctx->profiling && st != nullptr && st != cudaStreamLegacy;
+  bool use_graph = ctx->graph_cache && st != nullptr && st != cudaStreamLegacy;
   if (use_graph) {
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) { cudaGetLastError(); use_graph = false; }
   }
+  // A profiled forward is captured too, with the event records around its kernels as graph nodes, launched once and
+  // not cached: the kernels are then timed as they run inside a graph, not with a stream launch between the events.
+  const bool prof_graph = use_graph && ctx->profiling;
   std::string key;
-  if (use_graph) {
+  if (prof_graph) {
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); use_graph = false; }
+    else ctx->prof_capture = true;
+  } else if (use_graph) {
     // field by field: the structs contain padding bytes whose content the caller does not control
     auto put = [&key](const void* ptr, size_t n) { key.append((const char*)ptr, n); };
     auto put_aq = [&](const mixaq_aq& q) { put(&q.bits, 4); put(&q.scale, 4); put(&q.inv_scale, 4); put(&q.zero_point, 4); };
@@ -765,6 +783,9 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   mixaq_status result = MIXAQ_OK;
   int total = 0, H = H0, W = W0, blk = 0;
   const float* cur = x0;
+  // while profiling: a few event pairs with nothing between them, so that what a bracket itself adds to every kernel's
+  // time can be read off the same record
+  if (ctx->profiling) for (int i = 0; i < 4; ++i) { PROF(PC_BRACKET); }
   if (p->embed) {
     // image -> token map of stage 1 (patch embedding), inside the same captured graph
     result = mixaq_embed_forward(ctx, p->embed, x0, ws.tokens, B, Hi, Wi, ws.embed, ws.embed_bytes, st);
@@ -833,6 +854,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   if (use_graph) {
     cudaGraph_t graph = nullptr;
     cudaError_t e = cudaStreamEndCapture(st, &graph);
+    ctx->prof_capture = false;
     if (result != MIXAQ_OK) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return result; }
     cudaGraphExec_t exec = nullptr;
     if (e != cudaSuccess || !graph || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
@@ -841,8 +863,12 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
                  ? fail(ctx, MIXAQ_CUDA_ERROR, "backbone_forward: graph capture failed") : MIXAQ_CUDA_ERROR;
     }
     cudaGraphDestroy(graph);
-    if (ctx->graphs.size() >= 16) { cudaGraphExecDestroy(ctx->graphs.front().exec); ctx->graphs.erase(ctx->graphs.begin()); }
-    ctx->graphs.push_back({key, exec, total});
+    if (prof_graph && ctx->profiling) {
+      ctx->prof_execs.push_back(exec);
+    } else {
+      if (ctx->graphs.size() >= 16) { cudaGraphExecDestroy(ctx->graphs.front().exec); ctx->graphs.erase(ctx->graphs.begin()); }
+      ctx->graphs.push_back({key, exec, total});
+    }
     if (cudaGraphLaunch(exec, st) != cudaSuccess) return check_cuda(ctx, "backbone_forward (graph launch)");
   }
   if (result != MIXAQ_OK) return result;
