@@ -122,6 +122,8 @@ def cmd_traffic(args):
     rec = {"kernel_source_digest": kernel_source_digest(), "bytes_per_step": per_cat, "launches_per_step": dict(launches),
            "source": os.path.basename(args.report),
            "how": "dram__bytes_read.sum + dram__bytes_write.sum summed over the GEMM launches of one forward (one ncu capture)"}
+    if args.command:
+        rec["command"] = args.command
     if args.fc1_outputs and fc1_inst:
         rec["fc1_warp_inst_per_32_outputs"] = round(fc1_inst / (args.fc1_outputs / 32.0), 2)
     data = {}
@@ -139,6 +141,7 @@ def main():
     a = sub.add_parser("metrics"); a.add_argument("report"); a.add_argument("metric", nargs="*"); a.set_defaults(fn=cmd_metrics)
     a = sub.add_parser("traffic"); a.add_argument("report"); a.add_argument("--workload", required=True)
     a.add_argument("--fc1-outputs", type=float, default=0.0, help="fc1 outputs (rows x hidden) of one forward")
+    a.add_argument("--command", default="", help="the full ncu command that produced the report (kept in the record)")
     a.set_defaults(fn=cmd_traffic)
     args = ap.parse_args()
     args.fn(args)
