@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo, int 
 // codes per lane, and the butterfly (offsets 16, 8, 4, 2, 1 on the partial index) becomes log2(G) exchanges
 // between lanes followed by a tree inside the lane -- the same additions in the same order.
 template <int NG, int G>
-__global__ void __launch_bounds__(256, 4) k_ln_quant_g(LnBranch hi, LnBranch lo, int blocks_hi) {
+__global__ void __launch_bounds__(256, (NG * (32 / G) > 24 ? 2 : 4)) k_ln_quant_g(LnBranch hi, LnBranch lo, int blocks_hi) {
   constexpr int C = NG * 32, P = 32 / G, ROWS = 32 / G;     // channels, partials per lane, rows per warp
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int j = lane % G, rw = lane / G;
@@ -255,6 +255,8 @@ void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t
     else if (C == 256 && min_bits * 4 >= 8) launch_ln_g<8, 8>(hi, lo, st);
     else done = false;
   }
+  // wide rows: 8 lanes per row pay at any batch size (a third of the instructions of one warp per row)
+  if (!done && C == 384) { launch_ln_g<12, 8>(hi, lo, st); done = true; }
   if (done) { ++g_launches; return; }
   switch (C / 32) {
     MIXAQ_LN_CASE(1, 8) MIXAQ_LN_CASE(2, 8) MIXAQ_LN_CASE(3, 8) MIXAQ_LN_CASE(4, 8) MIXAQ_LN_CASE(6, 4)
