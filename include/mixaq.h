@@ -40,6 +40,7 @@ typedef int mixaq_status;
 #define MIXAQ_CUDA_ERROR           (-4)  /* a CUDA runtime/driver call failed; see mixaq_last_error()     */
 #define MIXAQ_DEVICE_TIMEOUT       (-5)  /* a bounded wait inside a kernel ran out (status word)          */
 #define MIXAQ_INTERNAL             (-6)
+#define MIXAQ_WORKSPACE_OVERRUN    (-7)  /* a guard zone between two workspace buffers was overwritten     */
 
 typedef struct mixaq_ctx mixaq_ctx;
 
@@ -138,7 +139,8 @@ mixaq_status mixaq_create(mixaq_ctx** ctx, int device);
 mixaq_status mixaq_destroy(mixaq_ctx* ctx);
 /* Text of the last host-side error of this context (static storage, valid until the next call). */
 const char*  mixaq_last_error(const mixaq_ctx* ctx);
-/* Reads the device status word (synchronises `cuda_stream`): MIXAQ_OK or MIXAQ_DEVICE_TIMEOUT. */
+/* Reads the device status word (synchronises `cuda_stream`): MIXAQ_OK, MIXAQ_DEVICE_TIMEOUT, or
+ * MIXAQ_WORKSPACE_OVERRUN (see mixaq_set_workspace_guards; reported in preference to a time-out). */
 mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream);
 
 /* Clears the status word (asynchronous on the stream). */
@@ -268,6 +270,17 @@ mixaq_status mixaq_set_window_elevation(mixaq_ctx* ctx, int allow);
  * scores go to the high-precision branch in every block.  Off by default; the block call has the same switch in
  * mixaq_select_opts. */
 mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse);
+
+/* Debug aid against out-of-bounds writes.  Every buffer the library carves out of a caller's workspace is followed by
+ * a 256-byte guard zone (always; the *_workspace_bytes figures include them).  enabled = 1: mixaq_block_forward (also
+ * as part of mixaq_backbone_forward) writes a pattern into the zones of the block's workspace before its first kernel
+ * and compares them after its last; a difference raises the status word (MIXAQ_WORKSPACE_OVERRUN from
+ * mixaq_last_device_status).  Two small launches per block; off by default. */
+mixaq_status mixaq_set_workspace_guards(mixaq_ctx* ctx, int enabled);
+/* Self-test of that check on a caller's buffer (>= 2 KiB of device memory): two 256-byte buffers are carved out of
+ * it, their guard zones filled, and, with overrun = 1, one byte just past the second buffer is written (inside the
+ * caller's memory) before the zones are compared. */
+mixaq_status mixaq_selftest_workspace_guards(mixaq_ctx* ctx, void* buffer, size_t bytes, int overrun, void* cuda_stream);
 
 /* NVTX ranges for external tracers (off by default): every kernel family launched through this context is wrapped in
  * a host-side range named like its profiling category, and mixaq_backbone_forward adds one range per stage and per

@@ -24,11 +24,11 @@ EXPORTS = [
     "mixaq_profile_begin", "mixaq_profile_end", "mixaq_merge_forward_static", "mixaq_set_graph_cache",
     "mixaq_embed_prepared_bytes", "mixaq_embed_prepare", "mixaq_embed_workspace_bytes", "mixaq_embed_forward",
     "mixaq_norm_forward", "mixaq_profile_end_records", "mixaq_calibrate_block_workspace_bytes", "mixaq_calibrate_block",
-    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection", "mixaq_set_nvtx",
+    "mixaq_calibrate_merge_workspace_bytes", "mixaq_calibrate_merge", "mixaq_aq_from_range", "mixaq_clear_device_status", "mixaq_selftest_wait_timeout", "mixaq_measure_mma_peak", "mixaq_set_window_elevation", "mixaq_set_reverse_selection", "mixaq_set_nvtx", "mixaq_set_workspace_guards", "mixaq_selftest_workspace_guards",
 ]
 
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED_SHAPE", -3: "WORKSPACE_TOO_SMALL", -4: "CUDA_ERROR",
-          -5: "DEVICE_TIMEOUT", -6: "INTERNAL"}
+          -5: "DEVICE_TIMEOUT", -6: "INTERNAL", -7: "WORKSPACE_OVERRUN"}
 
 
 class MixaqError(RuntimeError):
@@ -161,6 +161,16 @@ class Context:
 
     def device_status(self) -> int:
         return lib().mixaq_last_device_status(self.h, _stream_ptr())
+
+    def set_workspace_guards(self, enabled: bool):
+        """mixaq_set_workspace_guards: fill / compare the guard zones of the block workspace around every block."""
+        self.check(lib().mixaq_set_workspace_guards(self.h, 1 if enabled else 0), "set_workspace_guards")
+
+    def selftest_workspace_guards(self, overrun: bool):
+        """mixaq_selftest_workspace_guards on a scratch buffer of this context's device."""
+        buf = torch.zeros(4096, dtype=torch.uint8, device=self.device)
+        self.check(lib().mixaq_selftest_workspace_guards(self.h, _ptr(buf), C.c_size_t(buf.numel()), 1 if overrun else 0,
+                                                         _stream_ptr()), "selftest_workspace_guards")
 
     def set_nvtx(self, enabled: bool):
         """mixaq_set_nvtx: host-side NVTX ranges per kernel family, stage and block."""

@@ -45,6 +45,11 @@ struct MergeGatherArgs {
   const float* x; const float *gamma, *beta; uint8_t* out; AQ q; int B, H, W, C;
 };
 void launch_merge_gather(const MergeGatherArgs& a, cudaStream_t st);
+// ---- guard zones of the workspaces (debug aid) -------------------------------------------------------
+constexpr int GUARD_BYTES = 256;          // after every buffer of a workspace
+// fill = true: writes the guard pattern into every zone; fill = false: compares, and on a difference sets bit 1 of *status
+void launch_guards(void* const* zones, int count, bool fill, int* status, cudaStream_t st);
+
 void launch_copy_rows(const float* x, float* y, const int32_t* rowsrc, int M, int C, cudaStream_t st);
 
 // ---- stem and output norms ---------------------------------------------------------------------------

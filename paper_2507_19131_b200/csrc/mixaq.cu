@@ -32,6 +32,7 @@ struct mixaq_ctx {
   bool reverse_selection;              // backbone: worst-case selection order (Table 4) in every block
   bool prof_capture;                   // the profiled call is being captured: event records become graph nodes
   std::vector<cudaGraphExec_t> prof_execs;   // graphs of profiled forwards, destroyed when the profiling ends
+  bool guards;                         // fill the guard zones of the workspace before a forward, compare them after it
   bool nvtx;                           // name every kernel family, stage and block with an NVTX range (host side)
   bool allow_elevation;                // backbone: every pair uses its own ratios even if an earlier pair of the stage had larger ones
   std::vector<GraphEntry> graphs;
@@ -60,10 +61,31 @@ namespace {
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
+// Every buffer carved out of a workspace is followed by a guard zone of GUARD_BYTES that no kernel has a reason to
+// touch.  With mixaq_set_workspace_guards the zones are filled with a pattern before a forward and compared after it.
+thread_local std::vector<void*>* t_guard_log = nullptr;     // where the carver notes its guard zones (NULL: nowhere)
 struct Carver {
-  char* base; size_t off;
-  explicit Carver(void* p) : base((char*)p), off(0) {}
-  template <class T> T* take(size_t n) { T* p = base ? (T*)(base + off) : nullptr; off += align_up(n * sizeof(T)); return p; }
+  char* base; size_t off; bool guarded;
+  // guarded = false: the `prepared` parameter tables, written once by the prepare calls (their layout is also read by
+  // code that does not carve)
+  explicit Carver(void* p, bool with_guards = true) : base((char*)p), off(0), guarded(with_guards) {}
+  template <class T> T* take(size_t n) {
+    T* p = base ? (T*)(base + off) : nullptr;
+    off += align_up(n * sizeof(T));
+    if (guarded) {
+      if (base && t_guard_log) t_guard_log->push_back(base + off);
+      off += GUARD_BYTES;
+    }
+    return p;
+  }
+};
+// bytes a guarded carver needs for one buffer of n bytes
+inline size_t carved_bytes(size_t n) { return align_up(n) + GUARD_BYTES; }
+// scope in which carvers log their guard zones into `list` (when the context asks for guards)
+struct GuardScope {
+  std::vector<void*>* prev;
+  GuardScope(const mixaq_ctx* ctx, std::vector<void*>* list) : prev(t_guard_log) { t_guard_log = (ctx && ctx->guards) ? list : nullptr; }
+  ~GuardScope() { t_guard_log = prev; }
 };
 
 AQ to_aq(const mixaq_aq& q) {
@@ -164,7 +186,7 @@ struct Prepared {
   float* mult[4][2]; int32_t* zc[4][2]; float* relbias; size_t bytes;
 };
 Prepared carve_prepared(const mixaq_block_params* p, void* base) {
-  Prepared r; Carver c(base);
+  Prepared r; Carver c(base, false);
   const int N[4] = {3 * p->dim, p->dim, p->hidden, p->dim};
   for (int l = 0; l < 4; ++l)
     for (int b = 0; b < 2; ++b) { r.mult[l][b] = c.take<float>(N[l]); r.zc[l][b] = c.take<int32_t>(N[l]); }
@@ -266,7 +288,7 @@ mixaq_status mixaq_create(mixaq_ctx** out, int device) {
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MIXAQ_CUDA_ERROR; }
   mixaq_ctx* c = new (std::nothrow) mixaq_ctx();
   if (!c) return MIXAQ_INTERNAL;
-  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false; c->nvtx = false; c->prof_capture = false;
+  c->device = device; c->launches = 0; c->err[0] = 0; c->d_status = nullptr; c->profiling = false; c->graph_cache = true; c->allow_elevation = false; c->reverse_selection = false; c->nvtx = false; c->prof_capture = false; c->guards = false;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess || cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
       !gemm_init()) {
     cudaGetLastError(); if (c->d_status) cudaFree(c->d_status); delete c; return MIXAQ_CUDA_ERROR;
@@ -296,7 +318,7 @@ mixaq_status mixaq_last_device_status(mixaq_ctx* ctx, void* cuda_stream) {
   if (cudaMemcpyAsync(&h, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess)
   { check_cuda(ctx, "status read"); return MIXAQ_CUDA_ERROR; }
-  return h == 0 ? MIXAQ_OK : MIXAQ_DEVICE_TIMEOUT;
+  return h == 0 ? MIXAQ_OK : ((h & 2) ? MIXAQ_WORKSPACE_OVERRUN : MIXAQ_DEVICE_TIMEOUT);
 }
 
 mixaq_status mixaq_clear_device_status(mixaq_ctx* ctx, void* cuda_stream) {
@@ -413,7 +435,7 @@ size_t mixaq_merge_prepared_bytes(const mixaq_merge_params* p) {
 mixaq_status mixaq_merge_prepare(mixaq_ctx* ctx, const mixaq_merge_params* p, void* cuda_stream) {
   if (!ctx || !p) return MIXAQ_INVALID_ARG;
   if (!p->prepared || !p->reduction.codes || !p->reduction.scale) return fail(ctx, MIXAQ_INVALID_ARG, "merge params incomplete");
-  Carver c(p->prepared);
+  Carver c(p->prepared, false);
   float* mult = c.take<float>(p->reduction.out_features);
   int32_t* zc = c.take<int32_t>(p->reduction.out_features);
   launch_prepare_linear(p->reduction.codes, p->reduction.scale, p->reduction.out_features, p->reduction.in_features,
@@ -454,11 +476,14 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   Geometry g = geometry(H, W, low_ratio, prune_ratio);
   if ((size_t)g.nW * 8 > 48 * 1024) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many windows per image (max 6144)");
   if (!workspace) return fail(ctx, MIXAQ_INVALID_ARG, "workspace is NULL");
-  BlockWs ws = carve_block(p, B, H, W, workspace);
+  std::vector<void*> guard_zones;
+  BlockWs ws;
+  { GuardScope gs(ctx, &guard_zones); ws = carve_block(p, B, H, W, workspace); }
   if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "workspace too small");
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const int C = p->dim, Hd = p->hidden;
   Prepared pr = carve_prepared(p, p->prepared);
+  if (!guard_zones.empty()) launch_guards(guard_zones.data(), (int)guard_zones.size(), true, ctx->d_status, st);
   g_launches = 0;
 
   // 1. scores and selection
@@ -574,6 +599,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
     }
   }
   ctx->launches = g_launches;
+  if (!guard_zones.empty()) launch_guards(guard_zones.data(), (int)guard_zones.size(), false, ctx->d_status, st);
   return check_cuda(ctx, "block_forward");
 }
 
@@ -612,7 +638,7 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
   mg.x = x; mg.gamma = p->ln_g; mg.beta = p->ln_b; mg.out = (uint8_t*)workspace; mg.q = to_aq(p->in);
   mg.B = B; mg.H = H; mg.W = W; mg.C = C;
   { PROF(PC_MERGE_GATHER); launch_merge_gather(mg, st); }
-  Carver c(p->prepared);
+  Carver c(p->prepared, false);
   float* mult = c.take<float>(N);
   int32_t* zc = c.take<int32_t>(N);
   GemmArgs ga;
@@ -882,7 +908,7 @@ namespace {
 constexpr int EMBED_K = 48, EMBED_KP = 64;     // patch vector, padded to a multiple of 32 codes
 struct EmbedPrepared { int8_t* w; float* mult; int32_t* zc; size_t bytes; };
 EmbedPrepared carve_embed(const mixaq_embed_params* p, void* base) {
-  EmbedPrepared r; Carver c(base);
+  EmbedPrepared r; Carver c(base, false);
   const int N = p->proj.out_features;
   r.w = c.take<int8_t>((size_t)N * EMBED_KP); r.mult = c.take<float>(N); r.zc = c.take<int32_t>(N);
   r.bytes = c.off;
@@ -914,7 +940,7 @@ mixaq_status mixaq_embed_prepare(mixaq_ctx* ctx, const mixaq_embed_params* p, vo
 size_t mixaq_embed_workspace_bytes(const mixaq_embed_params* p, int B, int Hi, int Wi) {
   if (!p || B <= 0 || Hi <= 0 || Wi <= 0 || p->proj.out_features <= 0) return 0;
   const size_t toks = (size_t)B * ((Hi + 3) / 4) * ((Wi + 3) / 4);
-  return align_up(toks * EMBED_KP) + align_up(toks * p->proj.out_features * sizeof(float));
+  return carved_bytes(toks * EMBED_KP) + carved_bytes(toks * p->proj.out_features * sizeof(float));
 }
 
 mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, const float* image, float* x0,
@@ -962,6 +988,33 @@ mixaq_status mixaq_set_reverse_selection(mixaq_ctx* ctx, int reverse) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   ctx->reverse_selection = reverse != 0;
   return MIXAQ_OK;
+}
+
+mixaq_status mixaq_set_workspace_guards(mixaq_ctx* ctx, int enabled) {
+  if (!ctx) return MIXAQ_INVALID_ARG;
+  ctx->guards = enabled != 0;
+  return MIXAQ_OK;
+}
+
+mixaq_status mixaq_selftest_workspace_guards(mixaq_ctx* ctx, void* buffer, size_t bytes, int overrun, void* cuda_stream) {
+  if (!ctx || !buffer || bytes < 4 * (size_t)(256 + GUARD_BYTES)) return MIXAQ_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  std::vector<void*> zones;
+  uint8_t* second = nullptr;
+  {
+    const bool was = ctx->guards;
+    ctx->guards = true;
+    GuardScope gs(ctx, &zones);
+    Carver c(buffer);
+    c.take<uint8_t>(256);
+    second = c.take<uint8_t>(256);
+    ctx->guards = was;
+  }
+  launch_guards(zones.data(), (int)zones.size(), true, ctx->d_status, st);
+  // a writer that runs one byte past the end of the second buffer (an ordinary write inside the caller's memory)
+  if (overrun) cudaMemsetAsync(second + 256, 0, 1, st);
+  launch_guards(zones.data(), (int)zones.size(), false, ctx->d_status, st);
+  return check_cuda(ctx, "selftest_workspace_guards");
 }
 
 mixaq_status mixaq_set_nvtx(mixaq_ctx* ctx, int enabled) {
@@ -1047,7 +1100,7 @@ mixaq_status mixaq_calibrate_block(mixaq_ctx* ctx, const mixaq_block_params* p, 
 size_t mixaq_calibrate_merge_workspace_bytes(const mixaq_merge_params* p, int B, int H, int W) {
   if (!p || B <= 0 || H <= 0 || W <= 0 || p->reduction.in_features <= 0) return 0;
   const size_t toks = (size_t)B * ((H + 1) / 2) * ((W + 1) / 2);
-  return align_up(16 * sizeof(uint32_t)) + align_up(toks * p->reduction.in_features * sizeof(float));
+  return carved_bytes(16 * sizeof(uint32_t)) + carved_bytes(toks * p->reduction.in_features * sizeof(float));
 }
 
 mixaq_status mixaq_calibrate_merge(mixaq_ctx* ctx, const mixaq_merge_params* p, const float* x, float* y,

@@ -151,4 +151,28 @@ void launch_select(const SelectArgs* args, int count, cudaStream_t st) {
   }
 }
 
+// ---- guard zones ---------------------------------------------------------------------------------------
+namespace {
+constexpr int GUARD_BATCH = 48;
+constexpr uint32_t GUARD_PATTERN = 0xA5C3E1B7u;
+struct GuardList { uint32_t* zone[GUARD_BATCH]; };
+template <bool FILL>
+__global__ void k_guards(GuardList g, int* status) {
+  uint32_t* z = g.zone[blockIdx.x];
+  const int i = threadIdx.x;                               // GUARD_BYTES / 4 threads
+  if (FILL) z[i] = GUARD_PATTERN ^ (uint32_t)i;
+  else if (z[i] != (GUARD_PATTERN ^ (uint32_t)i)) atomicOr(status, 2);
+}
+}  // namespace
+
+void launch_guards(void* const* zones, int count, bool fill, int* status, cudaStream_t st) {
+  for (int first = 0; first < count; first += GUARD_BATCH) {
+    const int n = count - first < GUARD_BATCH ? count - first : GUARD_BATCH;
+    GuardList g;
+    for (int i = 0; i < GUARD_BATCH; ++i) g.zone[i] = (uint32_t*)zones[first + (i < n ? i : 0)];
+    if (fill) k_guards<true><<<n, GUARD_BYTES / 4, 0, st>>>(g, status);
+    else k_guards<false><<<n, GUARD_BYTES / 4, 0, st>>>(g, status);
+  }
+}
+
 }  // namespace mixaq

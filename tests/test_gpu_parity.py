@@ -399,6 +399,38 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(orc, mq):
         c.close()
 
 
+def test_workspace_guard_zones(orc, mq):
+    """The guard zones behind every workspace buffer: untouched by a forward (block with all taps, and a small
+    backbone through its graph), and the check itself reports a byte written just past a buffer."""
+    c = mq.Context(0)
+    try:
+        c.set_workspace_guards(True)
+        blk = synth.make_block(np.random.default_rng(52), 64, 2, 3, 4, 8, 4)
+        x = synth.input_blobs(53, 2, 17, 23, 64, bg_std=0.5, gain=4.0)
+        run_block_case(orc, mq, c, blk, x, 0.4, 0.1)
+        assert c.device_status() == 0
+        wl = synth.tiny_backbone()
+        want = orc.backbone_forward(wl.backbone, wl.x, wl.low_ratios, wl.prune_ratios)
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            dbb = mq.DeviceBackbone(c, wl.backbone, wl.B, wl.H, wl.W)
+            xd = dev(wl.x)
+            for _ in range(2):
+                got = mq.backbone_forward(c, dbb, xd, wl.low_ratios, wl.prune_ratios)
+            side.synchronize()
+            for g, w in zip(got, want):
+                assert np.array_equal(g.cpu().numpy(), w)
+        assert c.device_status() == 0
+        c.selftest_workspace_guards(overrun=False)
+        assert c.device_status() == 0
+        c.selftest_workspace_guards(overrun=True)
+        assert c.device_status() == -7                       # MIXAQ_WORKSPACE_OVERRUN
+        c.clear_device_status()
+        assert c.device_status() == 0
+    finally:
+        c.close()
+
+
 def test_mma_issue_rate_microbenchmark(mq, ctx):
     """The library's own tensor-core loop: kind::i8 reaches petaops; kind::f8f6f4 (the path of the 4/6-bit operand
     formats in 8-bit containers) is not faster; kind::mxf4 (block-scaled E2M1, the one narrower path with a higher
