@@ -1,9 +1,9 @@
 """Turns Nsight Compute output into the short records kept under profiles/.
 
-  python -m paper_2507_19131_b200.ncu_summary launches gpurun_out/launches.csv
+  python -m paper_2507_19131_b200.ncu_summary launches out/launches.csv
       per kernel: launches, total time, share (from `ncu --metrics gpu__time_duration.sum --csv --log-file ...`)
 
-  python -m paper_2507_19131_b200.ncu_summary traffic gpurun_out/gemm_traffic.ncu-rep --workload cfg3-swin_t-800x1333 \
+  python -m paper_2507_19131_b200.ncu_summary traffic out/gemm_traffic.ncu-rep --workload cfg3-swin_t-800x1333 \
          --fc1-outputs 130351104
       DRAM bytes of the GEMM launches of ONE forward (the report must hold exactly the GEMM launches of one forward:
       `ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,smsp__inst_executed.sum -k regex:k_gemm_tc -c <n>`),
