@@ -16,6 +16,9 @@
  *   - Every pointer inside the *_params structs, x, y, stage outputs, selections, taps and workspaces is a
  *     DEVICE pointer owned by the caller.  The library never frees them and keeps none past the call, with
  *     one exception: `prepared` buffers are read by every later forward call that gets the same params.
+ *   - Alignment: feature maps, weight codes and LayerNorm parameters 16 bytes; workspaces and `prepared` buffers
+ *     256 bytes (what cudaMalloc and the usual framework allocators give).  Anything less is refused with
+ *     MIXAQ_INVALID_ARG before a launch.
  *   - Feature maps are [B][H][W][C] binary32, channels contiguous.  C must be a multiple of 32, C/heads
  *     must be 32, window must be 7, hidden must be a multiple of 32.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*); they allocate no device memory and do

@@ -60,6 +60,10 @@ static const char* kProfNames[PC_COUNT] = {"energy", "select", "gather_ln1_quant
 namespace {
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+// The kernels read and write feature maps, parameters and codes with 16-byte accesses and describe operand matrices
+// to the TMA unit (16-byte aligned base); workspaces and prepared buffers are carved in 256-byte steps.  A pointer
+// that breaks this would fault on the device, so it is refused on the host.
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // Every buffer carved out of a workspace is followed by a guard zone of GUARD_BYTES that no kernel has a reason to
 // touch.  With mixaq_set_workspace_guards the zones are filled with a pattern before a forward and compared after it.
@@ -171,6 +175,13 @@ mixaq_status validate_block(mixaq_ctx* ctx, const mixaq_block_params* p, bool ne
       !linear_ok(p->fc1, p->hidden, p->dim) || !linear_ok(p->fc2, p->dim, p->hidden))
     return fail(ctx, MIXAQ_INVALID_ARG, "weight matrix missing or of the wrong shape");
   if (!p->relpos_table) return fail(ctx, MIXAQ_INVALID_ARG, "relpos_table is NULL");
+  {
+    const void* q16[] = {p->qkv.codes, p->proj.codes, p->fc1.codes, p->fc2.codes,
+                         p->hi.ln1_g, p->hi.ln1_b, p->hi.ln2_g, p->hi.ln2_b, p->lo.ln1_g, p->lo.ln1_b, p->lo.ln2_g, p->lo.ln2_b};
+    for (const void* q : q16)
+      if (!aligned_to(q, 16)) return fail(ctx, MIXAQ_INVALID_ARG, "weight codes and LayerNorm parameters must be 16-byte aligned");
+    if (p->prepared && !aligned_to(p->prepared, 256)) return fail(ctx, MIXAQ_INVALID_ARG, "prepared buffer must be 256-byte aligned");
+  }
   if (p->byte_codes != 0 && p->byte_codes != 1) return fail(ctx, MIXAQ_INVALID_ARG, "byte_codes must be 0 or 1");
   if (!need_quantizers) {
     if (!branch_ptrs_ok(p->hi) || !branch_ptrs_ok(p->lo)) return fail(ctx, MIXAQ_INVALID_ARG, "branch parameters invalid");
@@ -468,6 +479,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   mixaq_status s = validate_block(ctx, p);
   if (s != MIXAQ_OK) return s;
   if (!x || !y || x == y) return fail(ctx, MIXAQ_INVALID_ARG, "x / y NULL or aliased");
+  if (!aligned_to(x, 16) || !aligned_to(y, 16)) return fail(ctx, MIXAQ_INVALID_ARG, "x and y must be 16-byte aligned");
   if (B <= 0 || H <= 0 || W <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "B, H, W must be positive");
   if (!(low_ratio >= 0.f && low_ratio <= 1.f) || !(prune_ratio >= 0.f && prune_ratio <= 1.f))
     return fail(ctx, MIXAQ_INVALID_ARG, "ratios must lie in [0, 1]");
@@ -476,6 +488,7 @@ static mixaq_status block_forward_impl(mixaq_ctx* ctx, const mixaq_block_params*
   Geometry g = geometry(H, W, low_ratio, prune_ratio);
   if ((size_t)g.nW * 8 > 48 * 1024) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many windows per image (max 6144)");
   if (!workspace) return fail(ctx, MIXAQ_INVALID_ARG, "workspace is NULL");
+  if (!aligned_to(workspace, 256)) return fail(ctx, MIXAQ_INVALID_ARG, "workspace must be 256-byte aligned");
   std::vector<void*> guard_zones;
   BlockWs ws;
   { GuardScope gs(ctx, &guard_zones); ws = carve_block(p, B, H, W, workspace); }
@@ -625,6 +638,9 @@ mixaq_status mixaq_merge_forward(mixaq_ctx* ctx, const mixaq_merge_params* p, co
                                  int B, int H, int W, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!ctx || !p) return MIXAQ_INVALID_ARG;
   if (!x || !y || !workspace || B <= 0 || H <= 0 || W <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "merge: bad argument");
+  if (!aligned_to(x, 16) || !aligned_to(y, 16) || !aligned_to(workspace, 256) || !aligned_to(p->prepared, 256) ||
+      !aligned_to(p->reduction.codes, 16) || !aligned_to(p->ln_g, 16) || !aligned_to(p->ln_b, 16))
+    return fail(ctx, MIXAQ_INVALID_ARG, "merge: x, y, weights and LayerNorm parameters must be 16-byte aligned, workspace and prepared 256-byte");
   const int K = p->reduction.in_features, N = p->reduction.out_features, C = K / 4;
   if (K % 4 || N % 32 || !merge_dim_supported(C)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "merge: unsupported dims");
   if (!p->ln_g || !p->ln_b || !p->reduction.codes || !p->reduction.scale || !p->prepared || !bits_ok(p->in.bits) ||
@@ -712,6 +728,8 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
     return fail(ctx, MIXAQ_INVALID_ARG, "backbone params incomplete");
   if (!x0 || !stage_out || !low_ratio_per_pair || !workspace || B <= 0 || H0 <= 0 || W0 <= 0)
     return fail(ctx, MIXAQ_INVALID_ARG, "backbone: bad argument");
+  if (!aligned_to(x0, 16) || !aligned_to(workspace, 256))
+    return fail(ctx, MIXAQ_INVALID_ARG, "backbone: x0 must be 16-byte aligned, the workspace 256-byte");
   if (p->num_stages > 16) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "at most 16 stages");
   if ((p->out_norm_g != nullptr) != (p->out_norm_b != nullptr)) return fail(ctx, MIXAQ_INVALID_ARG, "output norms need gamma and beta");
   const bool norms = p->out_norm_g && p->out_norm_b;
@@ -727,6 +745,7 @@ mixaq_status mixaq_backbone_forward(mixaq_ctx* ctx, const mixaq_backbone_params*
   for (int s = 0; s < p->num_stages; ++s) {
     if (p->depths[s] <= 0 || (p->depths[s] != 1 && p->depths[s] % 2)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "depths must be even or 1");
     if (!stage_out[s]) return fail(ctx, MIXAQ_INVALID_ARG, "stage_out entry is NULL");
+    if (!aligned_to(stage_out[s], 16)) return fail(ctx, MIXAQ_INVALID_ARG, "stage_out entries must be 16-byte aligned");
     nblk += p->depths[s];
   }
   for (int b = 0; b < nblk; ++b) {

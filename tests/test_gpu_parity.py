@@ -468,4 +468,18 @@ def test_invalid_arguments_are_rejected_before_any_launch(mq, ctx):
                                C.c_float(0.5), C.c_float(0.0), None, None, C.c_void_p(ws.data_ptr()),
                                C.c_size_t(ws.numel()), None, None)
     assert st == -2
+    # pointers the kernels could only touch with misaligned accesses are refused on the host: x off by 4 bytes,
+    # workspace off by 16, a weight matrix off by 1
+    big = torch.zeros(x.numel() + 4, device="cuda")
+    for xp, wp in ((big.data_ptr() + 4, ws.data_ptr()), (x.data_ptr(), ws.data_ptr() + 16)):
+        st = L.mixaq_block_forward(ctx.h, C.byref(db.s), C.c_void_p(xp), C.c_void_p(y.data_ptr()), 1, 14, 14,
+                                   C.c_float(0.5), C.c_float(0.0), None, None, C.c_void_p(wp),
+                                   C.c_size_t(ws.numel() - 16), None, None)
+        assert st == -1
+    bad = mq.BlockS.from_buffer_copy(db.s)
+    bad.fc1.codes = bad.fc1.codes + 1
+    st = L.mixaq_block_forward(ctx.h, C.byref(bad), C.c_void_p(x.data_ptr()), C.c_void_p(y.data_ptr()), 1, 14, 14,
+                               C.c_float(0.5), C.c_float(0.0), None, None, C.c_void_p(ws.data_ptr()),
+                               C.c_size_t(ws.numel()), None, None)
+    assert st == -1
     assert ctx.device_status() == 0
