@@ -457,6 +457,7 @@ mixaq_status mixaq_merge_prepare(mixaq_ctx* ctx, const mixaq_merge_params* p, vo
 mixaq_status mixaq_stage_energy(mixaq_ctx* ctx, const float* x, int32_t* energy, int B, int H, int W, int C,
                                 float score_inv_scale, void* cuda_stream) {
   if (!ctx || !x || !energy || B <= 0 || H <= 0 || W <= 0 || C <= 0 || !(score_inv_scale > 0.f)) return MIXAQ_INVALID_ARG;
+  if (!aligned_to(x, 16) || !aligned_to(energy, 4)) return fail(ctx, MIXAQ_INVALID_ARG, "stage_energy: x must be 16-byte aligned");
   launch_energy(x, energy, (long)B * H * W, C, score_inv_scale, (cudaStream_t)cuda_stream);
   return check_cuda(ctx, "stage_energy");
 }
@@ -967,6 +968,9 @@ mixaq_status mixaq_embed_forward(mixaq_ctx* ctx, const mixaq_embed_params* p, co
   if (!ctx) return MIXAQ_INVALID_ARG;
   if (!embed_ok(p) || !p->prepared) return fail(ctx, MIXAQ_INVALID_ARG, "embed params incomplete");
   if (!image || !x0 || !workspace || B <= 0 || Hi <= 0 || Wi <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "embed: bad argument");
+  if (!aligned_to(image, 4) || !aligned_to(x0, 16) || !aligned_to(workspace, 256) || !aligned_to(p->prepared, 256) ||
+      !aligned_to(p->ln_g, 16) || !aligned_to(p->ln_b, 16) || !aligned_to(p->bias, 16))
+    return fail(ctx, MIXAQ_INVALID_ARG, "embed: x0 and parameters must be 16-byte aligned, workspace and prepared 256-byte");
   if (mixaq_embed_workspace_bytes(p, B, Hi, Wi) > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "embed workspace");
   const size_t toks = (size_t)B * ((Hi + 3) / 4) * ((Wi + 3) / 4);
   if (toks >= (size_t)1 << 31) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many tokens");
@@ -996,6 +1000,8 @@ mixaq_status mixaq_norm_forward(mixaq_ctx* ctx, const float* gamma, const float*
                                 long rows, int C, void* cuda_stream) {
   if (!ctx) return MIXAQ_INVALID_ARG;
   if (!gamma || !beta || !x || !y || rows <= 0 || C <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "norm: bad argument");
+  if (!aligned_to(gamma, 16) || !aligned_to(beta, 16) || !aligned_to(x, 16) || !aligned_to(y, 16))
+    return fail(ctx, MIXAQ_INVALID_ARG, "norm: pointers must be 16-byte aligned");
   g_launches = 0;
   if (!launch_bias_ln(x, nullptr, gamma, beta, y, rows, C, (cudaStream_t)cuda_stream))
     return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "norm: unsupported C");
@@ -1096,6 +1102,8 @@ mixaq_status mixaq_calibrate_block(mixaq_ctx* ctx, const mixaq_block_params* p, 
   if (s != MIXAQ_OK) return s;
   if (!x || !y || x == y || !ranges || !workspace || B <= 0 || H <= 0 || W <= 0 || (branch != 0 && branch != 1))
     return fail(ctx, MIXAQ_INVALID_ARG, "calibrate_block: bad argument");
+  if (!aligned_to(x, 16) || !aligned_to(y, 16) || !aligned_to(workspace, 256))
+    return fail(ctx, MIXAQ_INVALID_ARG, "calibrate_block: x and y must be 16-byte aligned, the workspace 256-byte");
   if ((long)B * H * W >= (1L << 31) / WT) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "too many tokens");
   CalWs ws = carve_cal(p, B, H, W, workspace);
   if (ws.bytes > workspace_bytes) return fail(ctx, MIXAQ_WORKSPACE_TOO_SMALL, "calibrate_block workspace too small");
@@ -1127,6 +1135,8 @@ mixaq_status mixaq_calibrate_merge(mixaq_ctx* ctx, const mixaq_merge_params* p, 
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!ctx || !p) return MIXAQ_INVALID_ARG;
   if (!x || !y || !range || !workspace || B <= 0 || H <= 0 || W <= 0) return fail(ctx, MIXAQ_INVALID_ARG, "calibrate_merge: bad argument");
+  if (!aligned_to(x, 16) || !aligned_to(y, 16) || !aligned_to(workspace, 256) || !aligned_to(p->reduction.codes, 16))
+    return fail(ctx, MIXAQ_INVALID_ARG, "calibrate_merge: x, y and weights must be 16-byte aligned, the workspace 256-byte");
   const int K = p->reduction.in_features, N = p->reduction.out_features, C = K / 4;
   if (K % 4 || N <= 0 || !merge_dim_supported(C)) return fail(ctx, MIXAQ_UNSUPPORTED_SHAPE, "calibrate_merge: unsupported dims");
   if (!p->ln_g || !p->ln_b || !p->reduction.codes || !p->reduction.scale) return fail(ctx, MIXAQ_INVALID_ARG, "merge params incomplete");
