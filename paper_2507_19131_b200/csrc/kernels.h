@@ -38,6 +38,8 @@ struct LnBranch {
   uint8_t* out;              // [M][C*bits/8]
   AQ q;
   int M;
+  int mgH, mgW;              // patch merging only: size of the input map (row m is an OUTPUT token, its C channels are
+                             // those of the 2x2 input neighbours, C/4 each)
 };
 void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st);
 

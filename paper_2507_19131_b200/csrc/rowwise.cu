@@ -60,9 +60,13 @@ __global__ void __launch_bounds__(256) k_ln_quant(LnBranch hi, LnBranch lo, int 
 // partials, i.e. of every 32-channel group the P contiguous channels 32i + P*j ..: vector loads, whole bytes of
 // codes per lane, and the butterfly (offsets 16, 8, 4, 2, 1 on the partial index) becomes log2(G) exchanges
 // between lanes followed by a tree inside the lane -- the same additions in the same order.
-template <int NG, int G>
+// MERGE: the rows are the output tokens of a patch merging: channel group i of a row comes from input neighbour
+// i / (NG/4) (order (0,0), (1,0), (0,1), (1,1)); neighbours outside the map are zeros that take part in the LayerNorm.
+template <int NG, int G, bool MERGE>
 __global__ void __launch_bounds__(256, (NG * (32 / G) > 24 ? 2 : 4)) k_ln_quant_g(LnBranch hi, LnBranch lo, int blocks_hi) {
   constexpr int C = NG * 32, P = 32 / G, ROWS = 32 / G;     // channels, partials per lane, rows per warp
+  constexpr int VEC = P >= 4 ? 4 : 2;                       // floats per load
+  static_assert(P >= 2 && (!MERGE || NG % 4 == 0), "unsupported lane split");
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int j = lane % G, rw = lane / G;
   const bool is_hi = (int)blockIdx.x < blocks_hi;
@@ -75,16 +79,38 @@ __global__ void __launch_bounds__(256, (NG * (32 / G) > 24 ? 2 : 4)) k_ln_quant_
   const AQ q = br.q;
   const int bits = q.bits;
   long srow = -1;
-  if (m < M) srow = br.rowsrc ? (long)br.rowsrc[m] : (long)m;
+  if (m < M) srow = (MERGE || !br.rowsrc) ? (long)m : (long)br.rowsrc[m];
+  // source rows: one (gather / plain) or the four input neighbours (merge); -1: zeros
+  long nsrc[MERGE ? 4 : 1];
+  if (MERGE) {
+    const int H2 = (br.mgH + 1) / 2, W2 = (br.mgW + 1) / 2;
+    const int mm = m < M ? m : 0;
+    const int b = mm / (H2 * W2), r2 = mm - b * (H2 * W2), y2 = r2 / W2, x2 = r2 - y2 * W2;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const int yy = 2 * y2 + (g & 1), xx = 2 * x2 + (g >> 1);
+      nsrc[MERGE ? g : 0] = (m < M && yy < br.mgH && xx < br.mgW) ? ((long)b * br.mgH + yy) * br.mgW + xx : -1;
+    }
+  } else {
+    nsrc[0] = srow;
+  }
   float x[NG][P];
-  const float* row = br.src + (srow < 0 ? 0 : srow) * C + P * j;
 #pragma unroll
   for (int i = 0; i < NG; ++i) {
+    constexpr int GPN = MERGE ? NG / 4 : NG;                 // channel groups per source row
+    const long sr = nsrc[MERGE ? i / GPN : 0];
+    const float* src = br.src + (sr < 0 ? 0 : sr) * (GPN * 32) + 32 * (i % GPN) + P * j;
 #pragma unroll
-    for (int v4 = 0; v4 < P / 4; ++v4) {
-      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (srow >= 0) a = __ldg(reinterpret_cast<const float4*>(row + 32 * i) + v4);
-      x[i][4 * v4] = a.x; x[i][4 * v4 + 1] = a.y; x[i][4 * v4 + 2] = a.z; x[i][4 * v4 + 3] = a.w;
+    for (int v = 0; v < P / VEC; ++v) {
+      if (VEC == 4) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (sr >= 0) a = __ldg(reinterpret_cast<const float4*>(src) + v);
+        x[i][4 * v] = a.x; x[i][4 * v + 1] = a.y; x[i][4 * v + 2] = a.z; x[i][4 * v + 3] = a.w;
+      } else {
+        float2 a = make_float2(0.f, 0.f);
+        if (sr >= 0) a = __ldg(reinterpret_cast<const float2*>(src) + v);
+        x[i][2 * v] = a.x; x[i][2 * v + 1] = a.y;
+      }
     }
   }
   // partial sums in channel order, then the butterfly: lanes first (offsets 16 .. P), then inside the lane
@@ -137,13 +163,20 @@ __global__ void __launch_bounds__(256, (NG * (32 / G) > 24 ? 2 : 4)) k_ln_quant_
     for (int i = 0; i < NG; ++i) {
       uint32_t w0 = kpack, w1 = kpack;
 #pragma unroll
-      for (int v4 = 0; v4 < P / 4; ++v4) {
-        const float4 g4 = __ldg(reinterpret_cast<const float4*>(br.gamma + 32 * i + P * j) + v4);
-        const float4 b4 = __ldg(reinterpret_cast<const float4*>(br.beta + 32 * i + P * j) + v4);
-        const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
+      for (int v4 = 0; v4 < P / VEC; ++v4) {
+        float gg[4], bb[4];
+        if (VEC == 4) {
+          const float4 g4 = __ldg(reinterpret_cast<const float4*>(br.gamma + 32 * i + P * j) + v4);
+          const float4 b4 = __ldg(reinterpret_cast<const float4*>(br.beta + 32 * i + P * j) + v4);
+          gg[0] = g4.x; gg[1] = g4.y; gg[2] = g4.z; gg[3] = g4.w; bb[0] = b4.x; bb[1] = b4.y; bb[2] = b4.z; bb[3] = b4.w;
+        } else {
+          const float2 g2 = __ldg(reinterpret_cast<const float2*>(br.gamma + 32 * i + P * j) + v4);
+          const float2 b2 = __ldg(reinterpret_cast<const float2*>(br.beta + 32 * i + P * j) + v4);
+          gg[0] = g2.x; gg[1] = g2.y; gg[2] = gg[3] = 0.f; bb[0] = b2.x; bb[1] = b2.y; bb[2] = bb[3] = 0.f;
+        }
 #pragma unroll
-        for (int e = 0; e < 4; e += 2) {
-          const int k = 4 * v4 + e;
+        for (int e = 0; e < VEC; e += 2) {
+          const int k = VEC * v4 + e;
           // y = fma((x - mean) * rstd, gamma, beta) on two channels, then their magic patterns
           const float2 d = __fmul2_rn(sub2(make_float2(x[i][k], x[i][k + 1]), f2(mean)), f2(rstd));
           const float2 y = __ffma2_rn(d, make_float2(gg[e], gg[e + 1]), make_float2(bb[e], bb[e + 1]));
@@ -232,11 +265,11 @@ void launch_ln_npl(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
 }
 #define MIXAQ_LN_CASE(n, rmax) case n: launch_ln_npl<n, rmax>(hi, lo, st); break;
 
-template <int NG, int G>
+template <int NG, int G, bool MERGE = false>
 void launch_ln_g(const LnBranch& hi, const LnBranch& lo, cudaStream_t st) {
   const int rpb = 8 * (32 / G);                              // rows per block: 8 warps x 32/G rows
   const int bh = (hi.M + rpb - 1) / rpb, bl = (lo.M + rpb - 1) / rpb;
-  k_ln_quant_g<NG, G><<<bh + bl, 256, 0, st>>>(hi, lo, bh);
+  k_ln_quant_g<NG, G, MERGE><<<bh + bl, 256, 0, st>>>(hi, lo, bh);
 }
 
 void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t st) {
@@ -257,6 +290,7 @@ void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t
   }
   // wide rows: 8 lanes per row pay at any batch size (a third of the instructions of one warp per row)
   if (!done && C == 384) { launch_ln_g<12, 8>(hi, lo, st); done = true; }
+  if (!done && C == 768 && min_bits * 2 >= 8) { launch_ln_g<24, 16>(hi, lo, st); done = true; }
   if (done) { ++g_launches; return; }
   switch (C / 32) {
     MIXAQ_LN_CASE(1, 8) MIXAQ_LN_CASE(2, 8) MIXAQ_LN_CASE(3, 8) MIXAQ_LN_CASE(4, 8) MIXAQ_LN_CASE(6, 4)
@@ -268,6 +302,17 @@ void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t
 
 void launch_merge_gather(const MergeGatherArgs& a, cudaStream_t st) {
   long toks = (long)a.B * ((a.H + 1) / 2) * ((a.W + 1) / 2);
+  // 4C = 384 / 768: the multi-lane LayerNorm kernel with the rows gathered from the four input neighbours
+  if ((4 * a.C == 384 || (4 * a.C == 768 && a.q.bits * 2 >= 8)) && toks < (1L << 31)) {
+    LnBranch hi, lo;
+    hi.src = a.x; hi.rowsrc = nullptr; hi.gamma = a.gamma; hi.beta = a.beta; hi.out = a.out; hi.q = a.q; hi.M = (int)toks;
+    hi.mgH = a.H; hi.mgW = a.W;
+    lo = hi; lo.M = 0;
+    if (4 * a.C == 384) launch_ln_g<12, 8, true>(hi, lo, st);
+    else launch_ln_g<24, 16, true>(hi, lo, st);
+    ++g_launches;
+    return;
+  }
   unsigned grid = (unsigned)((toks + 7) / 8);
   switch (4 * a.C / 32) {
     MIXAQ_NPL_CASE(4, k_merge_gather, a) MIXAQ_NPL_CASE(8, k_merge_gather, a) MIXAQ_NPL_CASE(12, k_merge_gather, a)
