@@ -290,7 +290,9 @@ void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t
   }
   // wide rows: 8 lanes per row pay at any batch size (a third of the instructions of one warp per row)
   if (!done && C == 384) { launch_ln_g<12, 8>(hi, lo, st); done = true; }
+  if (!done && C == 512) { launch_ln_g<16, 8>(hi, lo, st); done = true; }
   if (!done && C == 768 && min_bits * 2 >= 8) { launch_ln_g<24, 16>(hi, lo, st); done = true; }
+  if (!done && C == 1024 && min_bits * 2 >= 8) { launch_ln_g<32, 16>(hi, lo, st); done = true; }
   if (done) { ++g_launches; return; }
   switch (C / 32) {
     MIXAQ_LN_CASE(1, 8) MIXAQ_LN_CASE(2, 8) MIXAQ_LN_CASE(3, 8) MIXAQ_LN_CASE(4, 8) MIXAQ_LN_CASE(6, 4)
@@ -302,14 +304,17 @@ void launch_ln_quant(const LnBranch& hi, const LnBranch& lo, int C, cudaStream_t
 
 void launch_merge_gather(const MergeGatherArgs& a, cudaStream_t st) {
   long toks = (long)a.B * ((a.H + 1) / 2) * ((a.W + 1) / 2);
-  // 4C = 384 / 768: the multi-lane LayerNorm kernel with the rows gathered from the four input neighbours
-  if ((4 * a.C == 384 || (4 * a.C == 768 && a.q.bits * 2 >= 8)) && toks < (1L << 31)) {
+  // 4C = 384 ... 1024: the multi-lane LayerNorm kernel with the rows gathered from the four input neighbours
+  const int K4 = 4 * a.C;
+  if ((K4 == 384 || K4 == 512 || ((K4 == 768 || K4 == 1024) && a.q.bits * 2 >= 8)) && toks < (1L << 31)) {
     LnBranch hi, lo;
     hi.src = a.x; hi.rowsrc = nullptr; hi.gamma = a.gamma; hi.beta = a.beta; hi.out = a.out; hi.q = a.q; hi.M = (int)toks;
     hi.mgH = a.H; hi.mgW = a.W;
     lo = hi; lo.M = 0;
-    if (4 * a.C == 384) launch_ln_g<12, 8, true>(hi, lo, st);
-    else launch_ln_g<24, 16, true>(hi, lo, st);
+    if (K4 == 384) launch_ln_g<12, 8, true>(hi, lo, st);
+    else if (K4 == 512) launch_ln_g<16, 8, true>(hi, lo, st);
+    else if (K4 == 768) launch_ln_g<24, 16, true>(hi, lo, st);
+    else launch_ln_g<32, 16, true>(hi, lo, st);
     ++g_launches;
     return;
   }

@@ -139,7 +139,7 @@ def test_block_degenerate_splits(orc, mq, ctx, low, prune):
 def test_block_single_window_and_wide_dims(orc, mq, ctx):
     blk = synth.make_block(np.random.default_rng(30), 32, 1, 0, 8, 8, 4)
     run_block_case(orc, mq, ctx, blk, synth.input_blobs(31, 1, 5, 6, 32), 0.0)
-    for dim in (128, 192, 384):
+    for dim in (128, 192, 384, 512, 768):
         blk = synth.make_block(np.random.default_rng(dim), dim, dim // 32, 3, 4, 8, 4)
         run_block_case(orc, mq, ctx, blk, synth.input_blobs(dim + 1, 1, 14, 15, dim, bg_std=0.5), 0.5)
 
